@@ -1,0 +1,242 @@
+/*
+ * marl_actor.h - C ABI of the batched decentralised actor step for multi-agent RL on one GPU.
+ *
+ * What the library does.  A "worker" in the actor-worker-learner framework (Sec. III-B, Algorithm 2)
+ * repeats: get the observations of all of its environments, decide with the shared policy network, send
+ * the actions back.  Each environment step is recorded and whole episodes are handed to the learner's
+ * replay pool (Algorithm 1; Algorithm 3, "store it in the experience replay pool").  The hidden state of
+ * the recurrent agent is kept per (environment, agent) and never mixed across environments (Sec. III-A,
+ * Fig. 3).  This library is that loop for E environments x n agents on the GPU:
+ *
+ *     x  = [obs | one-hot(agent) | one-hot(last action)]        (last action: none at episode start)
+ *     y  = relu(W1 x + b1)
+ *     h' = GRUCell(y, h)        r|z|n row blocks, h' = (1-z)*c + z*h, c = tanh(W_in y + b_in + r*(W_hn h + b_hn))
+ *     Q  = W2 h' + b2
+ *     greedy = lowest available a with Q[a] >= max_avail(Q) - 1e-4f
+ *     action = explore ? uniform pick among the available actions : greedy
+ *              (Philox4x32-10, counter (step, env, agent, 0), key = seed; explore iff u < eps)
+ *     ring[slot_e][pos_e] <- (obs, avail, action, Q, reward, done);  episode end or full slot -> next slot,
+ *              h <- 0, last action <- none.
+ *
+ * The paper names a value-based (Qmix) agent but prints neither its layers nor the exploration rule; the
+ * network, the tie rule and the random-number keying above are this library's definition.
+ *
+ * Conventions
+ *   - Every function returns MARL_OK (0) or a negative error code; marl_last_error() gives the text.
+ *     Nothing throws or aborts across this boundary.
+ *   - "device" pointers are CUDA device addresses on the device that was current at marl_actor_create;
+ *     "host" pointers are ordinary process memory.  Borrowed arrays must stay valid until the work
+ *     enqueued by the call has finished on the actor's stream; inputs are never written.
+ *   - All device work is enqueued on the stream given at creation and is asynchronous unless a function
+ *     says that it synchronises.
+ *   - Conditions detected on the device (a row with no available action, a bounded wait that expired, an
+ *     index out of range) set bits in a status word; a kernel never traps.
+ */
+#ifndef MARL_ACTOR_H
+#define MARL_ACTOR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MARL_OK 0
+#define MARL_EINVAL (-1) /* bad argument or configuration */
+#define MARL_EALIGN (-2) /* a buffer is not aligned as required (16 bytes) */
+#define MARL_ECUDA (-3)  /* a CUDA call failed; marl_last_error() names it */
+#define MARL_ENOMEM (-4) /* a caller-provided buffer is too small, or an allocation failed */
+
+#define MARL_PRECISION_FP32 0 /* fp32 weights, fp32 FFMA arithmetic */
+#define MARL_PRECISION_BF16 1 /* weight matrices and matmul operands rounded to bf16 (RNE), fp32 accumulate */
+
+#define MARL_KERNEL_AUTO 0   /* tensor-core kernel where it is supported and the batch is large, else FFMA */
+#define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
+#define MARL_KERNEL_TENSOR 2 /* tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
+
+#define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
+#define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
+#define MARL_STATUS_BAD_INDEX 4u /* a ring or state index was out of range and the access was skipped */
+
+typedef struct marl_actor marl_actor_t; /* opaque; owned by the library; freed by marl_actor_destroy */
+
+/* Dimensions follow Table II of the paper: n agents, A actions, observation width D. */
+typedef struct {
+  int32_t n_envs;        /* E >= 1 */
+  int32_t n_agents;      /* n in [1, 32] */
+  int32_t obs_dim;       /* D in [1, 512] */
+  int32_t n_actions;     /* A in [1, 32] */
+  int32_t hidden;        /* H in {32, 64, 96, 128} */
+  int32_t ring_episodes; /* C: episode slots of the replay ring, a positive multiple of E */
+  int32_t ring_steps;    /* L: steps per slot; an episode reaching L steps is truncated */
+  int32_t precision;     /* MARL_PRECISION_* */
+  int32_t kernel;        /* MARL_KERNEL_* */
+  int32_t reserved;      /* must be 0 */
+  uint64_t seed;         /* Philox key of the exploration stream */
+  void* stream;          /* cudaStream_t, borrowed; NULL = the legacy default stream */
+  /* Device memory.  NULL = the library allocates with cudaMalloc and owns it.  Otherwise the caller's
+   * buffer is borrowed until marl_actor_destroy; it must be 256-byte aligned and at least as large as
+   * marl_actor_query_sizes reports. */
+  void* ring_mem;
+  size_t ring_bytes;
+  void* state_mem;
+  size_t state_bytes;
+  void* work_mem;    /* staging for marl_rollout / marl_actor_step_host; may be larger than the minimum: */
+  size_t work_bytes; /* marl_rollout stages as many steps per window as fit */
+} marl_actor_config_t;
+
+typedef struct {
+  size_t ring_bytes;          /* replay ring incl. slot headers */
+  size_t state_bytes;         /* recurrent state, counters, status word, packed weights */
+  size_t work_bytes_min;      /* staging for one environment step */
+  size_t work_bytes_per_step; /* staging per additional step of a rollout window */
+} marl_actor_sizes_t;
+
+/* Seeded synthetic environment that stands in for the simulator of Algorithm 1 (Env.step, Env.done).
+ * Every stream is a Philox4x32-10 block with counter (step, env, agent | block << 16, tag) and key = seed;
+ * tags: 1 done+reward, 2 availability, 3 observation.  A "24-bit threshold" T means: event iff
+ * (word >> 8) < T.
+ *   done    : word 0 of block 0 of (step, env, agent 0, tag 1) against done_thresh24.
+ *   reward  : blocks 1 and 2 of the same stream; the first twelve 16-bit half-words (low half first),
+ *             summed, minus 393210, times 2^-16 (an Irwin-Hall stand-in for N(0,1), exact in fp32).
+ *   avail   : action 0 always 1; action a > 0: word a%4 of block a/4 of (step, env, agent, tag 2) against
+ *             avail_thresh_first (a < avail_split) or avail_thresh_rest.
+ *   obs     : law 0: word d%4 of block d/4 of (step, env, agent, tag 3): ((w >> 8) - 2^23) * 2^-23;
+ *             law 1: blocks 2d and 2d+1, Irwin-Hall as for the reward, clamped to [-3, 3].
+ *             Typed feature blocks: with type_block_len > 0, agents [0, n_type0) are type 0 and the others
+ *             type 1; dims [start, start+len) belong to type 0, [start+len, start+2len) to type 1, and an
+ *             agent's obs is 0 in the other type's block. */
+typedef struct {
+  uint64_t seed;
+  int32_t obs_law;
+  uint32_t done_thresh24;
+  uint32_t avail_thresh_first;
+  uint32_t avail_thresh_rest;
+  int32_t avail_split;
+  int32_t n_type0;
+  int32_t type_block_start;
+  int32_t type_block_len;
+} marl_synth_env_t;
+
+/* Replay ring as the learner sees it.  One record per (slot, step) at
+ *   base + slot * slot_stride + step * step_stride,
+ * fields at the given byte offsets inside the record (each 16-byte aligned):
+ *   obs f32[n][D], avail u8[n][A], action i32[n], q f32[n][A] (raw network output, unmasked),
+ *   reward f32, done u8.
+ * Environment e owns slots e*S .. e*S+S-1 (S = slots_per_env); its k-th episode (k = 0, 1, ...) is written
+ * to slot e*S + k%S with id k*E + e.  Headers: slot_epid (-1 = never used), slot_len (steps written),
+ * slot_complete (1 once the episode has ended or was truncated at L steps; a truncated episode's last
+ * done flag is 0).  All pointers are device addresses, valid until marl_actor_destroy. */
+typedef struct {
+  void* base;
+  size_t slot_stride, step_stride;
+  size_t off_obs, off_avail, off_action, off_q, off_reward, off_done;
+  int32_t episodes, steps, slots_per_env, n_envs, n_agents, obs_dim, n_actions, reserved;
+  int64_t* slot_epid;
+  int32_t* slot_len;
+  uint8_t* slot_complete;
+} marl_ring_view_t;
+
+/* Recurrent state (device arrays) plus the global step counter (host value). */
+typedef struct {
+  float* h;             /* [E][n][H] */
+  int32_t* last_action; /* [E][n], -1 = none */
+  int32_t* slot;        /* [E] slot of the open episode */
+  int32_t* pos;         /* [E] next position in that slot */
+  int64_t* ep_count;    /* [E] episodes closed so far */
+  uint64_t step;        /* steps taken since creation / reset: Philox counter word 0 of the next step */
+} marl_state_view_t;
+
+typedef struct {
+  uint64_t agent_steps; /* rows processed */
+  uint64_t episodes;    /* episodes closed (done or truncated) */
+  uint64_t explored;    /* rows that took the random branch */
+  uint64_t no_avail;    /* rows without any available action */
+  uint64_t truncated;   /* episodes closed by the step limit */
+} marl_counters_t;
+
+/* Sizes of the three device buffers for a configuration (memory fields of cfg are ignored). */
+int marl_actor_query_sizes(const marl_actor_config_t* cfg, marl_actor_sizes_t* out);
+
+/* Creates an actor: validates cfg, carves the buffers, zeroes the state (h = 0, no last action, env e at
+ * slot e*S position 0, headers empty, step 0).  Weights are undefined until marl_actor_set_weights.
+ * Fails with MARL_ECUDA if no CUDA device is usable: there is no CPU path. */
+int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out);
+
+/* Loads the network (Algorithm 2: "get parameters from the shared memory pool").  HOST fp32 arrays in
+ * [out][in] layout, copied and repacked before the call returns to the caller's stream order:
+ *   W1 [H][D+n+A], b1 [H], W_ih [3H][H], b_ih [3H], W_hh [3H][H], b_hh [3H] (row blocks r|z|n),
+ *   W2 [A][H], b2 [A].  In bf16 precision the four matrices are rounded to bf16 (RNE); biases stay fp32.
+ * version is stored and returned by marl_actor_weights_version. */
+int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
+                           const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
+                           const float* b2, uint64_t version);
+uint64_t marl_actor_weights_version(const marl_actor_t* a);
+
+/* One decision step for all E environments (Algorithm 2, loop body) with recording (Algorithm 1).
+ * DEVICE inputs, dense: obs f32[E][n][D], avail u8[E][n][A] (non-zero = available), reward f32[E],
+ * done u8[E] - the outcome of this step's joint action, recorded with it.  actions_out i32[E][n] (device)
+ * may be NULL.  eps is this step's exploration rate. */
+int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                    const uint8_t* done, float eps, int32_t* actions_out);
+
+/* The same step with HOST buffers (the observation-action pipe of Algorithms 1 and 2 when the simulators
+ * run on the host): copies the four inputs to the device, runs the step, copies the actions back and
+ * SYNCHRONISES the stream before returning.  Pinned host memory makes the copies asynchronous. */
+int marl_actor_step_host(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                         const uint8_t* done, float eps, int32_t* actions_out);
+
+/* Writes n_steps steps of the synthetic environment, starting at step t0, into DEVICE arrays laid out
+ * [step][E]...: obs f32[n_steps][E][n][D], avail u8[n_steps][E][n][A], reward f32[n_steps][E],
+ * done u8[n_steps][E].  Each array must be 16-byte aligned. */
+int marl_env_generate(const marl_actor_t* a, const marl_synth_env_t* env, uint32_t t0, int32_t n_steps,
+                      float* obs, uint8_t* avail, float* reward, uint8_t* done);
+
+/* T steps on environment outputs already staged on the device in the layout of marl_env_generate.
+ * Step k uses eps = eps_start + (eps_end - eps_start) * min(t, N) / N with t = the global step index and
+ * N = anneal_steps (N <= 0: eps_start throughout), evaluated in double and rounded to fp32.
+ * Environments are independent, so the kernel may run all T steps of one tile of environments before the
+ * next tile; results are those of T calls of marl_actor_step. */
+int marl_rollout_staged(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                        const uint8_t* done, int32_t T, double eps_start, double eps_end,
+                        int32_t anneal_steps);
+
+/* T steps against the synthetic environment: generates windows of steps into the work buffer and runs
+ * marl_rollout_staged on each. */
+int marl_rollout(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double eps_start, double eps_end,
+                 int32_t anneal_steps);
+
+/* Optional per-step trace for verification: from the next step on, step k after this call writes its
+ * actions to actions[k][E][n] and its Q rows to q[k][E][n][A] (device; either may be NULL) while
+ * k < capacity_steps.  Pass NULL, NULL, 0 to switch it off. */
+int marl_actor_set_trace(marl_actor_t* a, int32_t* actions, float* q, int32_t capacity_steps);
+
+int marl_ring_view(const marl_actor_t* a, marl_ring_view_t* out);
+int marl_actor_get_state(const marl_actor_t* a, marl_state_view_t* out);
+/* Copies the five device arrays of *in into the actor (device-to-device, on the stream) and sets the step
+ * counter.  Together with the ring memory this is a checkpoint. */
+int marl_actor_set_state(marl_actor_t* a, const marl_state_view_t* in);
+
+/* SYNCHRONISES the stream, then reports and keeps the status bits and counters accumulated so far. */
+int marl_actor_status(marl_actor_t* a, uint32_t* device_status, marl_counters_t* counters);
+
+/* Back to the state after creation (weights are kept).  Asynchronous. */
+int marl_actor_reset(marl_actor_t* a);
+
+/* SYNCHRONISES the stream and frees what the library allocated. */
+void marl_actor_destroy(marl_actor_t* a);
+
+/* Name of the step kernel in use: "ffma" or "tcgen05". */
+const char* marl_actor_kernel_name(const marl_actor_t* a);
+
+/* Launches of library kernels enqueued by this actor since creation (all kernels, all entry points). */
+uint64_t marl_actor_launch_count(const marl_actor_t* a);
+
+/* Text of the last error on the calling thread ("" if none). */
+const char* marl_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARL_ACTOR_H */

@@ -177,6 +177,22 @@ def select_action(q, avail, eps: float, seed: int, t: int, e: int, i: int):
     return int(a), int(ex.value), float(u.value), int(na.value)
 
 
+def select_batch(q, avail, eps, seed: int, t, e, i):
+    """Row-wise select_action: q [N][A], avail [N][A], eps/t/e/i [N] -> (action [N], explore [N])."""
+    q = _c(q, np.float32)
+    avail = _c(avail, np.uint8)
+    N, A = q.shape
+    eps = _c(np.broadcast_to(eps, (N,)), np.float32)
+    t = _c(np.broadcast_to(t, (N,)), np.uint32)
+    e = _c(np.broadcast_to(e, (N,)), np.uint32)
+    i = _c(np.broadcast_to(i, (N,)), np.uint32)
+    act = np.zeros(N, np.int32)
+    ex = np.zeros(N, np.uint8)
+    lib().oracle_select_batch(_ptr(q), _ptr(avail), C.c_int32(A), C.c_int64(N), _ptr(eps), C.c_uint64(seed),
+                              _ptr(t), _ptr(e), _ptr(i), _ptr(act), _ptr(ex))
+    return act, ex
+
+
 @dataclass
 class Session:
     """State, replay-pool image and counters of the oracle for a list of environments."""

@@ -355,6 +355,19 @@ int32_t oracle_select_action(const float* q, const uint8_t* avail, int32_t A, fl
   return first_avail;
 }
 
+// The same choice for N independent rows (a plain loop over oracle_select_action).
+//   q [N][A], avail [N][A], eps [N], t/e/i [N]  ->  action [N], explore [N]
+void oracle_select_batch(const float* q, const uint8_t* avail, int32_t A, int64_t N, const float* eps,
+                         uint64_t seed, const uint32_t* t, const uint32_t* e, const uint32_t* i,
+                         int32_t* action, uint8_t* explore) {
+  for (int64_t r = 0; r < N; ++r) {
+    uint8_t ex = 0;
+    action[r] = oracle_select_action(q + r * A, avail + r * A, A, eps[r], seed, t[r], e[r], i[r], &ex,
+                                     nullptr, nullptr);
+    if (explore) explore[r] = ex;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // State and ring initialisation for a list of environments.
 // ---------------------------------------------------------------------------------------------------

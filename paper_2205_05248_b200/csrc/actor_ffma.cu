@@ -1,0 +1,432 @@
+// CUDA-core (FFMA) actor kernel: any shape, fp32 or bf16-rounded operands with fp32 accumulation.
+//
+// One thread block owns a tile of whole environments (up to 64 agent rows) and runs all T steps of the
+// launch for that tile before taking the next tile: environments are independent (Sec. III-A, Fig. 3: one
+// hidden state per environment and agent), so the hidden state, the last actions and the ring cursors of
+// the tile stay in shared memory for the whole launch.  Per step the block runs the worker's decision
+// (Algorithm 2: observations in, policy network, actions out) and the actor's recording of the step
+// (Algorithm 1), in six phases separated by block barriers:
+//   A  stage obs (-> shared, and verbatim into the ring record), availability masks, open slot headers
+//   B  fc1 + one-hot column gathers + ReLU                       (register-tiled 4 rows x 4 columns)
+//   C  GRU cell: both gate GEMMs, gate math, new hidden state    (same tiling, 64 accumulators)
+//   D  fc2
+//   E  masked greedy choice, epsilon draw, ring/trace writes     (one thread per row)
+//   F  reward/done, episode bookkeeping, hidden-state reset      (one thread per environment)
+// Weights are read through the read-only path from k-major copies, so a warp's load of four output
+// columns for one k is one contiguous 256-byte segment.
+#include "common.cuh"
+
+namespace marl {
+
+constexpr int FF_RMAX = 64;      // rows per tile
+constexpr int FF_THREADS = 256;
+constexpr int FF_QSTRIDE = 33;   // row stride of the Q tile (odd: one row per thread without conflicts)
+
+struct FfmaSmem {
+  int Dp, Hp;
+  size_t off_xs, off_ys, off_hs, off_hq, off_qs, off_mask, off_la, off_env, total;
+};
+
+__host__ __device__ inline FfmaSmem ffma_smem_layout(int D, int H, int prec) {
+  FfmaSmem s;
+  int Dp = (D + 3) & ~3;
+  if ((Dp & 31) == 0) Dp += 4;
+  s.Dp = Dp;
+  s.Hp = H + 4;
+  size_t o = 0;
+  s.off_xs = o; o += sizeof(float) * FF_RMAX * s.Dp;
+  s.off_ys = o; o += sizeof(float) * FF_RMAX * s.Hp;
+  s.off_hs = o; o += sizeof(float) * 2 * FF_RMAX * s.Hp;
+  s.off_hq = s.off_hs;  // fp32 precision: the operand copy is the state itself
+  if (prec == MARL_PRECISION_BF16) { s.off_hq = o; o += sizeof(float) * 2 * FF_RMAX * s.Hp; }
+  s.off_qs = o; o += sizeof(float) * FF_RMAX * FF_QSTRIDE;
+  s.off_mask = o; o += sizeof(uint32_t) * FF_RMAX;
+  s.off_la = o; o += sizeof(int32_t) * FF_RMAX;
+  s.off_env = o; o += 32 * FF_RMAX;  // per-environment scratch: see EnvSlot
+  s.total = o;
+  return s;
+}
+
+struct EnvSlot {            // 32 bytes per environment of the tile
+  long long epc;
+  int32_t slot, pos;
+  float reward;
+  int32_t done;             // this step's done flag
+  int32_t ok;               // cursor was in range at tile load
+  int32_t reset;            // episode closed this step
+};
+
+__device__ __forceinline__ float sigmoid_accurate(float x) { return 1.0f / (1.0f + expf(-x)); }
+
+__global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_constant__ ActorParams p) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  const FfmaSmem sl = ffma_smem_layout(p.D, p.H, p.prec);
+  float* xs = reinterpret_cast<float*>(smem + sl.off_xs);
+  float* ys = reinterpret_cast<float*>(smem + sl.off_ys);
+  float* hs = reinterpret_cast<float*>(smem + sl.off_hs);
+  float* hq = reinterpret_cast<float*>(smem + sl.off_hq);  // == hs in fp32 precision
+  float* qs = reinterpret_cast<float*>(smem + sl.off_qs);
+  uint32_t* masks = reinterpret_cast<uint32_t*>(smem + sl.off_mask);
+  int32_t* la = reinterpret_cast<int32_t*>(smem + sl.off_la);
+  EnvSlot* envs = reinterpret_cast<EnvSlot*>(smem + sl.off_env);
+
+  const int tid = threadIdx.x;
+  const int n = p.n, D = p.D, A = p.A, H = p.H, Dp = sl.Dp, Hp = sl.Hp, H3 = 3 * p.H;
+  const bool lowp = p.prec == MARL_PRECISION_BF16;
+  const int hbuf = FF_RMAX * Hp;  // floats per hidden buffer
+  const int tx = tid & 15, ty = tid >> 4;
+
+  unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
+  uint32_t st_bits = 0;
+
+  for (int i = tid; i < (int)(sl.total / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;
+  __syncthreads();
+
+  for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+    const int e0 = tile * p.ept;
+    const int ne = min(p.ept, p.E - e0);  // environments in this tile
+    const int R = ne * n;                 // live rows
+    int cur = 0;
+
+    // ---- tile load: hidden state, last actions, ring cursors ----
+    for (int idx = tid; idx < R * H; idx += FF_THREADS) {
+      const int r = idx / H, j = idx - r * H;
+      const float v = p.h[(size_t)e0 * n * H + idx];
+      hs[r * Hp + j] = v;
+      if (lowp) hq[r * Hp + j] = bf16_round(v);
+    }
+    for (int r = tid; r < FF_RMAX; r += FF_THREADS) la[r] = (r < R) ? p.last_action[e0 * n + r] : -1;
+    if (tid < ne) {
+      EnvSlot s;
+      s.slot = p.slot[e0 + tid];
+      s.pos = p.pos[e0 + tid];
+      s.epc = p.ep_count[e0 + tid];
+      s.reward = 0.f;
+      s.done = 0;
+      s.reset = 0;
+      s.ok = (s.slot >= 0 && s.slot < p.E * p.S && s.pos >= 0 && s.pos < p.L) ? 1 : 0;
+      if (!s.ok) st_bits |= MARL_STATUS_BAD_INDEX;
+      envs[tid] = s;
+    }
+    __syncthreads();
+
+    for (int s = 0; s < p.T; ++s) {
+      const uint32_t t = p.t0 + (uint32_t)s;
+      const float eps = eps_at(p, t);
+      const int nxt = cur ^ 1;
+
+      // ---- phase A ----
+      {
+        const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
+        const int nD = n * D;
+        for (int idx = tid; idx < R * D; idx += FF_THREADS) {
+          const int r = idx / D, d = idx - r * D;
+          const int el = idx / nD;
+          const float v = src[idx];
+          xs[r * Dp + d] = lowp ? bf16_round(v) : v;
+          const EnvSlot& es = envs[el];
+          if (es.ok) {
+            float* dst = reinterpret_cast<float*>(p.ring + (size_t)es.slot * p.slot_stride +
+                                                  (size_t)es.pos * p.rl.rec_bytes + p.rl.off_obs);
+            dst[idx - el * nD] = v;
+          }
+        }
+        if (tid < R) {
+          const int el = tid / n, ai = tid - el * n;
+          const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + ((size_t)e0 * n + tid) * A;
+          const EnvSlot& es = envs[el];
+          uint8_t* dst = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes +
+                         p.rl.off_avail + ai * A;
+          uint32_t m = 0;
+          for (int a = 0; a < A; ++a) {
+            const uint8_t b = av[a];
+            if (b) m |= 1u << a;
+            if (es.ok) dst[a] = b ? 1 : 0;
+          }
+          masks[tid] = m;
+        }
+        if (tid < ne) {
+          EnvSlot& es = envs[tid];
+          es.reward = p.reward[(size_t)s * p.env_step_stride + e0 + tid];
+          es.done = p.done[(size_t)s * p.env_step_stride + e0 + tid] ? 1 : 0;
+          es.reset = 0;
+          if (es.ok && es.pos == 0) {  // an episode opens in this slot
+            p.slot_epid[es.slot] = es.epc * (long long)p.E + (e0 + tid);
+            p.slot_len[es.slot] = 0;
+            p.slot_complete[es.slot] = 0;
+          }
+        }
+      }
+      __syncthreads();
+
+      // ---- phase B: fc1 ----
+      for (int jb = 0; jb < H; jb += 64) {
+        const int j0 = jb + tx * 4;
+        float acc[4][4];
+        {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(p.b1 + j0));
+#pragma unroll
+          for (int m = 0; m < 4; ++m) { acc[m][0] = b.x; acc[m][1] = b.y; acc[m][2] = b.z; acc[m][3] = b.w; }
+        }
+        const int K4 = (D + 3) & ~3;
+        for (int k = 0; k < K4; k += 4) {
+          float4 xv[4];
+#pragma unroll
+          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xs + (ty + 16 * m) * Dp + k);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const float4 w = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(k + kk) * H + j0));
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+              const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
+              acc[m][0] = fmaf(xk, w.x, acc[m][0]);
+              acc[m][1] = fmaf(xk, w.y, acc[m][1]);
+              acc[m][2] = fmaf(xk, w.z, acc[m][2]);
+              acc[m][3] = fmaf(xk, w.w, acc[m][3]);
+            }
+          }
+        }
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int r = ty + 16 * m;
+          const int ai = r % n;
+          const float4 wid = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(D + ai) * H + j0));
+          float4 o = make_float4(acc[m][0] + wid.x, acc[m][1] + wid.y, acc[m][2] + wid.z, acc[m][3] + wid.w);
+          const int last = la[r];
+          if (last >= 0) {
+            const float4 wl = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(D + n + last) * H + j0));
+            o.x += wl.x; o.y += wl.y; o.z += wl.z; o.w += wl.w;
+          }
+          o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
+          if (lowp) { o.x = bf16_round(o.x); o.y = bf16_round(o.y); o.z = bf16_round(o.z); o.w = bf16_round(o.w); }
+          *reinterpret_cast<float4*>(ys + r * Hp + j0) = o;
+        }
+      }
+      __syncthreads();
+
+      // ---- phase C: GRU cell ----
+      for (int jb = 0; jb < H; jb += 64) {
+        const int j0 = jb + tx * 4;
+        float ar[4][4], az[4][4], ai_[4][4], ah[4][4];
+        {
+          const float4 bir = __ldg(reinterpret_cast<const float4*>(p.bih + j0));
+          const float4 biz = __ldg(reinterpret_cast<const float4*>(p.bih + H + j0));
+          const float4 bin = __ldg(reinterpret_cast<const float4*>(p.bih + 2 * H + j0));
+          const float4 bhr = __ldg(reinterpret_cast<const float4*>(p.bhh + j0));
+          const float4 bhz = __ldg(reinterpret_cast<const float4*>(p.bhh + H + j0));
+          const float4 bhn = __ldg(reinterpret_cast<const float4*>(p.bhh + 2 * H + j0));
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            ar[m][0] = bir.x + bhr.x; ar[m][1] = bir.y + bhr.y; ar[m][2] = bir.z + bhr.z; ar[m][3] = bir.w + bhr.w;
+            az[m][0] = biz.x + bhz.x; az[m][1] = biz.y + bhz.y; az[m][2] = biz.z + bhz.z; az[m][3] = biz.w + bhz.w;
+            ai_[m][0] = bin.x; ai_[m][1] = bin.y; ai_[m][2] = bin.z; ai_[m][3] = bin.w;
+            ah[m][0] = bhn.x; ah[m][1] = bhn.y; ah[m][2] = bhn.z; ah[m][3] = bhn.w;
+          }
+        }
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+          const float* act = pass == 0 ? ys : (hq + cur * hbuf);
+          const float* WT = pass == 0 ? p.WihT : p.WhhT;
+          for (int k = 0; k < H; k += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int m = 0; m < 4; ++m) v[m] = *reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const float* wrow = WT + (size_t)(k + kk) * H3 + j0;
+              const float4 wr = __ldg(reinterpret_cast<const float4*>(wrow));
+              const float4 wz = __ldg(reinterpret_cast<const float4*>(wrow + H));
+              const float4 wn = __ldg(reinterpret_cast<const float4*>(wrow + 2 * H));
+#pragma unroll
+              for (int m = 0; m < 4; ++m) {
+                const float a = kk == 0 ? v[m].x : kk == 1 ? v[m].y : kk == 2 ? v[m].z : v[m].w;
+                ar[m][0] = fmaf(a, wr.x, ar[m][0]); ar[m][1] = fmaf(a, wr.y, ar[m][1]);
+                ar[m][2] = fmaf(a, wr.z, ar[m][2]); ar[m][3] = fmaf(a, wr.w, ar[m][3]);
+                az[m][0] = fmaf(a, wz.x, az[m][0]); az[m][1] = fmaf(a, wz.y, az[m][1]);
+                az[m][2] = fmaf(a, wz.z, az[m][2]); az[m][3] = fmaf(a, wz.w, az[m][3]);
+                if (pass == 0) {
+                  ai_[m][0] = fmaf(a, wn.x, ai_[m][0]); ai_[m][1] = fmaf(a, wn.y, ai_[m][1]);
+                  ai_[m][2] = fmaf(a, wn.z, ai_[m][2]); ai_[m][3] = fmaf(a, wn.w, ai_[m][3]);
+                } else {
+                  ah[m][0] = fmaf(a, wn.x, ah[m][0]); ah[m][1] = fmaf(a, wn.y, ah[m][1]);
+                  ah[m][2] = fmaf(a, wn.z, ah[m][2]); ah[m][3] = fmaf(a, wn.w, ah[m][3]);
+                }
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int r = ty + 16 * m;
+          const float4 hp = *reinterpret_cast<const float4*>(hs + cur * hbuf + r * Hp + j0);
+          const float hpv[4] = {hp.x, hp.y, hp.z, hp.w};
+          float o[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float rg = sigmoid_accurate(ar[m][c]);
+            const float zg = sigmoid_accurate(az[m][c]);
+            const float cand = tanhf(fmaf(rg, ah[m][c], ai_[m][c]));
+            o[c] = fmaf(zg, hpv[c] - cand, cand);  // (1 - z) * cand + z * h
+          }
+          *reinterpret_cast<float4*>(hs + nxt * hbuf + r * Hp + j0) = make_float4(o[0], o[1], o[2], o[3]);
+          if (lowp)
+            *reinterpret_cast<float4*>(hq + nxt * hbuf + r * Hp + j0) =
+                make_float4(bf16_round(o[0]), bf16_round(o[1]), bf16_round(o[2]), bf16_round(o[3]));
+        }
+      }
+      __syncthreads();
+
+      // ---- phase D: fc2 (four threads per row, actions striped over them) ----
+      {
+        const int r = tid >> 2, part = tid & 3;
+        float acc[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const int a = part + 4 * m;
+          acc[m] = a < A ? __ldg(p.b2 + a) : 0.f;
+        }
+        const float* hv = hq + nxt * hbuf + r * Hp;
+        for (int k = 0; k < H; k += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(hv + k);
+#pragma unroll
+          for (int m = 0; m < 8; ++m) {
+            const int a = part + 4 * m;
+            if (a < A) {
+              const float4 w = __ldg(reinterpret_cast<const float4*>(p.W2 + (size_t)a * H + k));
+              acc[m] = fmaf(v.x, w.x, acc[m]);
+              acc[m] = fmaf(v.y, w.y, acc[m]);
+              acc[m] = fmaf(v.z, w.z, acc[m]);
+              acc[m] = fmaf(v.w, w.w, acc[m]);
+            }
+          }
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const int a = part + 4 * m;
+          if (a < A) qs[r * FF_QSTRIDE + a] = acc[m];
+        }
+      }
+      __syncthreads();
+
+      // ---- phase E: choice and recording, one thread per row ----
+      if (tid < R) {
+        const int el = tid / n, ai = tid - el * n;
+        const int e = e0 + el;
+        const float* qrow = qs + tid * FF_QSTRIDE;
+        uint32_t flags;
+        const int act = select_action([&](int a) { return qrow[a]; }, A, masks[tid], eps, p.seed, t,
+                                      (uint32_t)e, (uint32_t)ai, flags);
+        c_steps += 1;
+        c_explore += flags & 1u;
+        if (flags & 2u) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
+        la[tid] = act;
+        const EnvSlot& es = envs[el];
+        if (es.ok) {
+          uint8_t* rec = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes;
+          float* qd = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
+          for (int a = 0; a < A; ++a) qd[a] = qrow[a];
+          reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
+        }
+        const int tk = p.trace_first + s;
+        if (tk < p.trace_cap) {
+          const size_t grow = ((size_t)tk * p.E + e) * n + ai;
+          if (p.trace_actions) p.trace_actions[grow] = act;
+          if (p.trace_q)
+            for (int a = 0; a < A; ++a) p.trace_q[grow * A + a] = qrow[a];
+        }
+        if (p.actions_out && s == p.T - 1) p.actions_out[(size_t)e * n + ai] = act;
+      }
+      __syncthreads();  // the rows above read the cursors that the environment threads advance below
+      // ---- phase F (first half): reward/done and the episode cursor, one thread per environment ----
+      if (tid < ne) {
+        EnvSlot& es = envs[tid];
+        if (es.ok) {
+          uint8_t* rec = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes;
+          *reinterpret_cast<float*>(rec + p.rl.off_reward) = es.reward;
+          rec[p.rl.off_done] = (uint8_t)es.done;
+          const bool full = es.pos + 1 == p.L;
+          if (es.done || full) {
+            p.slot_len[es.slot] = es.pos + 1;
+            p.slot_complete[es.slot] = 1;
+            c_episodes += 1;
+            if (!es.done) c_trunc += 1;
+            es.epc += 1;
+            es.slot = (e0 + tid) * p.S + (int)(es.epc % p.S);
+            es.pos = 0;
+            es.reset = 1;
+          } else {
+            es.pos += 1;
+          }
+        }
+      }
+      __syncthreads();
+      // ---- phase F (second half): a closed episode starts from a zero hidden state and no last action ----
+      for (int idx = tid; idx < R * H; idx += FF_THREADS) {
+        const int r = idx / H, j = idx - r * H;
+        if (envs[r / n].reset) {
+          hs[nxt * hbuf + r * Hp + j] = 0.f;
+          if (lowp) hq[nxt * hbuf + r * Hp + j] = 0.f;
+        }
+      }
+      if (tid < R && envs[tid / n].reset) la[tid] = -1;
+      cur = nxt;
+      __syncthreads();
+    }
+
+    // ---- tile store ----
+    for (int idx = tid; idx < R * H; idx += FF_THREADS) {
+      const int r = idx / H, j = idx - r * H;
+      p.h[(size_t)e0 * n * H + idx] = hs[cur * hbuf + r * Hp + j];
+    }
+    if (tid < R) p.last_action[e0 * n + tid] = la[tid];
+    if (tid < ne) {
+      const EnvSlot& es = envs[tid];
+      if (es.ok) {
+        p.slot[e0 + tid] = es.slot;
+        p.pos[e0 + tid] = es.pos;
+        p.ep_count[e0 + tid] = es.epc;
+        if (es.pos > 0) p.slot_len[es.slot] = es.pos;
+      }
+    }
+    __syncthreads();
+  }
+
+  if (c_steps) atomicAdd(p.counters + CNT_AGENT_STEPS, c_steps);
+  if (c_explore) atomicAdd(p.counters + CNT_EXPLORED, c_explore);
+  if (c_noavail) atomicAdd(p.counters + CNT_NO_AVAIL, c_noavail);
+  if (c_episodes) atomicAdd(p.counters + CNT_EPISODES, c_episodes);
+  if (c_trunc) atomicAdd(p.counters + CNT_TRUNCATED, c_trunc);
+  if (st_bits) atomicOr(p.status, st_bits);
+}
+
+// Environments per tile and number of tiles for this kernel.
+void ffma_tiling(int E, int n, int sms, int* ept, int* num_tiles) {
+  int per = FF_RMAX / n;
+  if (per < 1) per = 1;
+  int spread = (E + sms - 1) / sms;  // small batches: one tile per SM before tiles grow
+  if (spread < 1) spread = 1;
+  if (per > spread) per = spread;
+  *ept = per;
+  *num_tiles = (E + per - 1) / per;
+}
+
+size_t ffma_smem_bytes(int D, int H, int prec) { return ffma_smem_layout(D, H, prec).total; }
+
+// Returns the number of kernels launched or a negative cudaError.
+int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream) {
+  const size_t smem = ffma_smem_bytes(p.D, p.H, p.prec);
+  static size_t configured = 0;
+  if (smem > configured) {
+    const cudaError_t e =
+        cudaFuncSetAttribute(actor_ffma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return -(int)e;
+    configured = smem;
+  }
+  int grid = p.num_tiles < sms ? p.num_tiles : sms;
+  if (grid < 1) grid = 1;
+  actor_ffma_kernel<<<grid, FF_THREADS, smem, stream>>>(p);
+  const cudaError_t err = cudaGetLastError();
+  return err == cudaSuccess ? 1 : -(int)err;
+}
+
+}  // namespace marl

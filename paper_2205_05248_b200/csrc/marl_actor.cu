@@ -1,0 +1,634 @@
+// Host runtime and C ABI of the actor library: configuration checks, buffer carving, weight repacking,
+// launch planning and the entry points declared in include/marl_actor.h.  All arithmetic of the actor
+// step runs in the kernels (actor_ffma.cu, actor_tc.cu, env_kernel.cu); nothing here computes on the CPU
+// and there is no CPU fallback.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+namespace marl {
+int launch_env_generate(const marl_synth_env_t& env, int E, int n, int D, int A, uint32_t t0, int n_steps,
+                        float* obs, uint8_t* avail, float* reward, uint8_t* done, int sms, cudaStream_t stream);
+void ffma_tiling(int E, int n, int sms, int* ept, int* num_tiles);
+size_t ffma_smem_bytes(int D, int H, int prec);
+int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream);
+// tensor-core kernel
+bool tc_supported(int n, int D, int A, int H, int prec);
+size_t tc_wpack_bytes(int n, int D, int A, int H);
+void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b1, const float* Wih,
+                     const float* bih, const float* Whh, const float* bhh, const float* W2, const float* b2,
+                     void* dst_host);
+void tc_tiling(int E, int n, int sms, int* ept, int* num_tiles);
+int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream);
+}  // namespace marl
+
+using namespace marl;
+
+static thread_local std::string g_err;
+
+static int fail(int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+#define CU_TRY(call)                                                                              \
+  do {                                                                                            \
+    const cudaError_t e_ = (call);                                                                \
+    if (e_ != cudaSuccess) return fail(MARL_ECUDA, "%s: %s", #call, cudaGetErrorString(e_));      \
+  } while (0)
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Carve {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  }
+};
+
+struct FfmaWeightOffsets { size_t W1T, b1, WihT, bih, WhhT, bhh, W2, b2, total; };
+
+static FfmaWeightOffsets ffma_weight_offsets(int n, int D, int A, int H) {
+  const int I = D + n + A;
+  FfmaWeightOffsets w;
+  Carve c;
+  w.W1T = c.take(sizeof(float) * (size_t)(I + 4) * H);
+  w.b1 = c.take(sizeof(float) * H);
+  w.WihT = c.take(sizeof(float) * (size_t)H * 3 * H);
+  w.bih = c.take(sizeof(float) * 3 * H);
+  w.WhhT = c.take(sizeof(float) * (size_t)H * 3 * H);
+  w.bhh = c.take(sizeof(float) * 3 * H);
+  w.W2 = c.take(sizeof(float) * (size_t)A * H);
+  w.b2 = c.take(sizeof(float) * 32);
+  w.total = c.off;
+  return w;
+}
+
+struct StateOffsets { size_t h, last_action, slot, pos, ep_count, counters, status, wff, wpack, total; };
+struct RingOffsets { size_t records, epid, len, complete, total; };
+struct WorkOffsets { size_t obs, avail, reward, done, actions, total; };
+
+static RecordLayout record_layout(int n, int D, int A) {
+  RecordLayout r;
+  size_t o = 0;
+  r.off_obs = (uint32_t)o; o = align_up(o + sizeof(float) * n * D, 16);
+  r.off_avail = (uint32_t)o; o = align_up(o + (size_t)n * A, 16);
+  r.off_action = (uint32_t)o; o = align_up(o + sizeof(int32_t) * n, 16);
+  r.off_q = (uint32_t)o; o = align_up(o + sizeof(float) * n * A, 16);
+  r.off_reward = (uint32_t)o;
+  r.off_done = (uint32_t)o + 4;
+  o += 16;
+  r.rec_bytes = (uint32_t)o;
+  r.pad = 0;
+  return r;
+}
+
+static StateOffsets state_offsets(const marl_actor_config_t& c) {
+  StateOffsets s;
+  Carve cv;
+  const size_t rows = (size_t)c.n_envs * c.n_agents;
+  s.h = cv.take(sizeof(float) * rows * c.hidden);
+  s.last_action = cv.take(sizeof(int32_t) * rows);
+  s.slot = cv.take(sizeof(int32_t) * c.n_envs);
+  s.pos = cv.take(sizeof(int32_t) * c.n_envs);
+  s.ep_count = cv.take(sizeof(int64_t) * c.n_envs);
+  s.counters = cv.take(sizeof(uint64_t) * CNT_N);
+  s.status = cv.take(sizeof(uint32_t) * 4);
+  s.wff = cv.take(ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
+  s.wpack = cv.take(tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden));
+  s.total = cv.off;
+  return s;
+}
+
+static RingOffsets ring_offsets(const marl_actor_config_t& c) {
+  RingOffsets r;
+  Carve cv;
+  const RecordLayout rl = record_layout(c.n_agents, c.obs_dim, c.n_actions);
+  r.records = cv.take((size_t)c.ring_episodes * c.ring_steps * rl.rec_bytes);
+  r.epid = cv.take(sizeof(int64_t) * c.ring_episodes);
+  r.len = cv.take(sizeof(int32_t) * c.ring_episodes);
+  r.complete = cv.take((size_t)c.ring_episodes);
+  r.total = cv.off;
+  return r;
+}
+
+// Staging of W steps of environment output plus one step of actions.
+static WorkOffsets work_offsets(const marl_actor_config_t& c, size_t W) {
+  WorkOffsets w;
+  Carve cv;
+  const size_t rows = (size_t)c.n_envs * c.n_agents;
+  w.obs = cv.take(sizeof(float) * rows * c.obs_dim * W);
+  w.avail = cv.take(rows * c.n_actions * W);
+  w.reward = cv.take(sizeof(float) * c.n_envs * W);
+  w.done = cv.take((size_t)c.n_envs * W);
+  w.actions = cv.take(sizeof(int32_t) * rows);
+  w.total = cv.off;
+  return w;
+}
+
+static int check_config(const marl_actor_config_t* c) {
+  if (!c) return fail(MARL_EINVAL, "config is NULL");
+  if (c->n_envs < 1) return fail(MARL_EINVAL, "n_envs must be >= 1");
+  if (c->n_agents < 1 || c->n_agents > 32) return fail(MARL_EINVAL, "n_agents must be in [1, 32]");
+  if (c->obs_dim < 1 || c->obs_dim > 512) return fail(MARL_EINVAL, "obs_dim must be in [1, 512]");
+  if (c->n_actions < 1 || c->n_actions > 32) return fail(MARL_EINVAL, "n_actions must be in [1, 32]");
+  if (c->hidden != 64 && c->hidden != 128) return fail(MARL_EINVAL, "hidden must be 64 or 128");
+  if (c->ring_steps < 1) return fail(MARL_EINVAL, "ring_steps must be >= 1");
+  if (c->ring_episodes < c->n_envs || c->ring_episodes % c->n_envs != 0)
+    return fail(MARL_EINVAL, "ring_episodes must be a positive multiple of n_envs");
+  if (c->precision != MARL_PRECISION_FP32 && c->precision != MARL_PRECISION_BF16)
+    return fail(MARL_EINVAL, "unknown precision");
+  if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR) return fail(MARL_EINVAL, "unknown kernel");
+  if (c->reserved != 0) return fail(MARL_EINVAL, "reserved must be 0");
+  if ((double)c->n_envs * c->n_agents > 1.0e9) return fail(MARL_EINVAL, "n_envs * n_agents too large");
+  return MARL_OK;
+}
+
+struct marl_actor {
+  marl_actor_config_t cfg;
+  cudaStream_t stream;
+  int device, sms;
+  bool use_tc;
+  uint8_t *ring, *state, *work;
+  bool own_ring, own_state, own_work;
+  size_t work_bytes;
+  StateOffsets so;
+  RingOffsets ro;
+  FfmaWeightOffsets wo;
+  RecordLayout rl;
+  uint64_t step;
+  uint64_t weights_version;
+  bool have_weights;
+  int32_t* trace_actions;
+  float* trace_q;
+  int32_t trace_cap, trace_next;
+  uint64_t launches;
+  std::vector<uint8_t> host_pack;
+};
+
+__global__ void init_state_kernel(int E, int n, int H, int S, int C, float* h, int32_t* la, int32_t* slot,
+                                  int32_t* pos, long long* epc, long long* epid, int32_t* len,
+                                  uint8_t* complete, unsigned long long* counters, uint32_t* status) {
+  const long long rows = (long long)E * n;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long i0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  for (long long i = i0; i < rows * H; i += stride) h[i] = 0.f;
+  for (long long i = i0; i < rows; i += stride) la[i] = -1;
+  for (long long i = i0; i < E; i += stride) {
+    slot[i] = (int32_t)(i * S);
+    pos[i] = 0;
+    epc[i] = 0;
+  }
+  for (long long i = i0; i < C; i += stride) {
+    epid[i] = -1;
+    len[i] = 0;
+    complete[i] = 0;
+  }
+  if (i0 < CNT_N) counters[i0] = 0;
+  if (i0 == 0) *status = 0;
+}
+
+static int enqueue_reset(marl_actor* a) {
+  const marl_actor_config_t& c = a->cfg;
+  uint8_t* st = a->state;
+  init_state_kernel<<<a->sms * 4, 256, 0, a->stream>>>(
+      c.n_envs, c.n_agents, c.hidden, c.ring_episodes / c.n_envs, c.ring_episodes,
+      reinterpret_cast<float*>(st + a->so.h), reinterpret_cast<int32_t*>(st + a->so.last_action),
+      reinterpret_cast<int32_t*>(st + a->so.slot), reinterpret_cast<int32_t*>(st + a->so.pos),
+      reinterpret_cast<long long*>(st + a->so.ep_count), reinterpret_cast<long long*>(a->ring + a->ro.epid),
+      reinterpret_cast<int32_t*>(a->ring + a->ro.len), a->ring + a->ro.complete,
+      reinterpret_cast<unsigned long long*>(st + a->so.counters), reinterpret_cast<uint32_t*>(st + a->so.status));
+  CU_TRY(cudaGetLastError());
+  a->launches += 1;
+  a->step = 0;
+  a->trace_next = 0;
+  return MARL_OK;
+}
+
+extern "C" {
+
+const char* marl_last_error(void) { return g_err.c_str(); }
+
+int marl_actor_query_sizes(const marl_actor_config_t* cfg, marl_actor_sizes_t* out) {
+  const int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!out) return fail(MARL_EINVAL, "out is NULL");
+  out->ring_bytes = ring_offsets(*cfg).total;
+  out->state_bytes = state_offsets(*cfg).total;
+  out->work_bytes_min = work_offsets(*cfg, 1).total;
+  out->work_bytes_per_step = work_offsets(*cfg, 2).total - work_offsets(*cfg, 1).total + 4 * 256;
+  return MARL_OK;
+}
+
+int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!out) return fail(MARL_EINVAL, "out is NULL");
+  *out = nullptr;
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CU_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10)
+    return fail(MARL_ECUDA, "device %s has compute capability %d.%d; this library is built for sm_100a only",
+                prop.name, prop.major, prop.minor);
+  marl_actor* a = new (std::nothrow) marl_actor();
+  if (!a) return fail(MARL_ENOMEM, "out of host memory");
+  a->cfg = *cfg;
+  a->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
+  a->device = dev;
+  a->sms = prop.multiProcessorCount;
+  a->so = state_offsets(*cfg);
+  a->ro = ring_offsets(*cfg);
+  a->wo = ffma_weight_offsets(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden);
+  a->rl = record_layout(cfg->n_agents, cfg->obs_dim, cfg->n_actions);
+  a->ring = a->state = a->work = nullptr;
+  a->own_ring = a->own_state = a->own_work = false;
+  a->step = 0;
+  a->weights_version = 0;
+  a->have_weights = false;
+  a->trace_actions = nullptr;
+  a->trace_q = nullptr;
+  a->trace_cap = a->trace_next = 0;
+  a->launches = 0;
+
+  const bool tc_ok = tc_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
+  if (cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) {
+    delete a;
+    return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
+  }
+  // Small batches leave most SMs without a 128-row tile: the FFMA kernel spreads them better.
+  a->use_tc = cfg->kernel == MARL_KERNEL_TENSOR ||
+              (cfg->kernel == MARL_KERNEL_AUTO && tc_ok && (long long)cfg->n_envs * cfg->n_agents >= 128LL * a->sms);
+
+  auto bind = [&](void* mem, size_t have, size_t need, uint8_t** dst, bool* own, const char* what) -> int {
+    if (mem) {
+      if (reinterpret_cast<uintptr_t>(mem) % 256) return fail(MARL_EALIGN, "%s must be 256-byte aligned", what);
+      if (have < need) return fail(MARL_ENOMEM, "%s: %zu bytes given, %zu needed", what, have, need);
+      *dst = static_cast<uint8_t*>(mem);
+      *own = false;
+    } else {
+      void* p = nullptr;
+      const cudaError_t e = cudaMalloc(&p, need);
+      if (e != cudaSuccess) return fail(MARL_ENOMEM, "cudaMalloc(%zu) for %s: %s", need, what, cudaGetErrorString(e));
+      *dst = static_cast<uint8_t*>(p);
+      *own = true;
+    }
+    return MARL_OK;
+  };
+  const size_t work_min = work_offsets(*cfg, 1).total;
+  rc = bind(cfg->ring_mem, cfg->ring_bytes, a->ro.total, &a->ring, &a->own_ring, "ring_mem");
+  if (!rc) rc = bind(cfg->state_mem, cfg->state_bytes, a->so.total, &a->state, &a->own_state, "state_mem");
+  if (!rc) {
+    a->work_bytes = cfg->work_mem ? cfg->work_bytes : work_min;
+    rc = bind(cfg->work_mem, cfg->work_bytes, work_min, &a->work, &a->own_work, "work_mem");
+  }
+  if (!rc) rc = enqueue_reset(a);
+  if (rc) {
+    const std::string keep = g_err;
+    if (a->own_ring && a->ring) cudaFree(a->ring);
+    if (a->own_state && a->state) cudaFree(a->state);
+    if (a->own_work && a->work) cudaFree(a->work);
+    delete a;
+    g_err = keep;
+    return rc;
+  }
+  *out = a;
+  return MARL_OK;
+}
+
+void marl_actor_destroy(marl_actor_t* a) {
+  if (!a) return;
+  cudaStreamSynchronize(a->stream);
+  if (a->own_ring) cudaFree(a->ring);
+  if (a->own_state) cudaFree(a->state);
+  if (a->own_work) cudaFree(a->work);
+  delete a;
+}
+
+static float to_bf16_value(float v) {
+  uint32_t u;
+  memcpy(&u, &v, 4);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return v;
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  u &= 0xFFFF0000u;
+  memcpy(&v, &u, 4);
+  return v;
+}
+
+int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
+                           const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
+                           const float* b2, uint64_t version) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a weight pointer is NULL");
+  const int n = a->cfg.n_agents, D = a->cfg.obs_dim, A = a->cfg.n_actions, H = a->cfg.hidden;
+  const int I = D + n + A;
+  const bool lowp = a->cfg.precision == MARL_PRECISION_BF16;
+  const size_t tcb = tc_wpack_bytes(n, D, A, H);
+  // The previous upload may still be in flight from this staging buffer.
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  a->host_pack.assign(a->wo.total + tcb, 0);
+  uint8_t* hp = a->host_pack.data();
+  auto q = [lowp](float v) { return lowp ? to_bf16_value(v) : v; };
+  float* W1T = reinterpret_cast<float*>(hp + a->wo.W1T);
+  for (int j = 0; j < H; ++j)
+    for (int k = 0; k < I; ++k) W1T[(size_t)k * H + j] = q(W1[(size_t)j * I + k]);
+  float* WihT = reinterpret_cast<float*>(hp + a->wo.WihT);
+  float* WhhT = reinterpret_cast<float*>(hp + a->wo.WhhT);
+  for (int r = 0; r < 3 * H; ++r)
+    for (int k = 0; k < H; ++k) {
+      WihT[(size_t)k * 3 * H + r] = q(W_ih[(size_t)r * H + k]);
+      WhhT[(size_t)k * 3 * H + r] = q(W_hh[(size_t)r * H + k]);
+    }
+  float* W2p = reinterpret_cast<float*>(hp + a->wo.W2);
+  for (int i = 0; i < A * H; ++i) W2p[i] = q(W2[i]);
+  memcpy(hp + a->wo.b1, b1, sizeof(float) * H);
+  memcpy(hp + a->wo.bih, b_ih, sizeof(float) * 3 * H);
+  memcpy(hp + a->wo.bhh, b_hh, sizeof(float) * 3 * H);
+  memcpy(hp + a->wo.b2, b2, sizeof(float) * A);
+  CU_TRY(cudaMemcpyAsync(a->state + a->so.wff, hp, a->wo.total, cudaMemcpyHostToDevice, a->stream));
+  if (tcb && tc_supported(n, D, A, H, a->cfg.precision)) {
+    tc_pack_weights(n, D, A, H, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, hp + a->wo.total);
+    CU_TRY(cudaMemcpyAsync(a->state + a->so.wpack, hp + a->wo.total, tcb, cudaMemcpyHostToDevice, a->stream));
+  }
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  a->weights_version = version;
+  a->have_weights = true;
+  return MARL_OK;
+}
+
+uint64_t marl_actor_weights_version(const marl_actor_t* a) { return a ? a->weights_version : 0; }
+
+static void fill_params(marl_actor* a, ActorParams& p) {
+  const marl_actor_config_t& c = a->cfg;
+  memset(&p, 0, sizeof(p));
+  p.E = c.n_envs; p.n = c.n_agents; p.D = c.obs_dim; p.A = c.n_actions; p.H = c.hidden;
+  p.I = c.obs_dim + c.n_agents + c.n_actions;
+  p.L = c.ring_steps;
+  p.S = c.ring_episodes / c.n_envs;
+  p.prec = c.precision;
+  p.seed = c.seed;
+  uint8_t* st = a->state;
+  const uint8_t* w = st + a->so.wff;
+  p.W1T = reinterpret_cast<const float*>(w + a->wo.W1T);
+  p.b1 = reinterpret_cast<const float*>(w + a->wo.b1);
+  p.WihT = reinterpret_cast<const float*>(w + a->wo.WihT);
+  p.bih = reinterpret_cast<const float*>(w + a->wo.bih);
+  p.WhhT = reinterpret_cast<const float*>(w + a->wo.WhhT);
+  p.bhh = reinterpret_cast<const float*>(w + a->wo.bhh);
+  p.W2 = reinterpret_cast<const float*>(w + a->wo.W2);
+  p.b2 = reinterpret_cast<const float*>(w + a->wo.b2);
+  p.wpack = st + a->so.wpack;
+  p.h = reinterpret_cast<float*>(st + a->so.h);
+  p.last_action = reinterpret_cast<int32_t*>(st + a->so.last_action);
+  p.slot = reinterpret_cast<int32_t*>(st + a->so.slot);
+  p.pos = reinterpret_cast<int32_t*>(st + a->so.pos);
+  p.ep_count = reinterpret_cast<long long*>(st + a->so.ep_count);
+  p.ring = a->ring + a->ro.records;
+  p.rl = a->rl;
+  p.slot_stride = (long long)c.ring_steps * a->rl.rec_bytes;
+  p.slot_epid = reinterpret_cast<long long*>(a->ring + a->ro.epid);
+  p.slot_len = reinterpret_cast<int32_t*>(a->ring + a->ro.len);
+  p.slot_complete = a->ring + a->ro.complete;
+  p.counters = reinterpret_cast<unsigned long long*>(st + a->so.counters);
+  p.status = reinterpret_cast<uint32_t*>(st + a->so.status);
+  p.trace_actions = a->trace_actions;
+  p.trace_q = a->trace_q;
+  p.trace_first = a->trace_next;
+  p.trace_cap = (a->trace_actions || a->trace_q) ? a->trace_cap : 0;
+}
+
+// Enqueues T steps reading inputs laid out [step][E]...; shared by every stepping entry point.
+static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, const float* reward,
+                         const uint8_t* done, int T, bool eps_const, float eps, double eps_start,
+                         double eps_end, int anneal, int32_t* actions_out) {
+  if (!a->have_weights) return fail(MARL_EINVAL, "marl_actor_set_weights has not been called");
+  if (a->step + (uint64_t)T > 0xFFFFFFFFull) return fail(MARL_EINVAL, "step counter would exceed 32 bits");
+  const marl_actor_config_t& c = a->cfg;
+  ActorParams p;
+  fill_params(a, p);
+  p.T = T;
+  p.t0 = (uint32_t)a->step;
+  p.eps_const_mode = eps_const ? 1 : 0;
+  p.eps_const = eps;
+  p.eps_start = eps_start;
+  p.eps_end = eps_end;
+  p.anneal_steps = anneal;
+  p.obs = obs; p.avail = avail; p.reward = reward; p.done = done;
+  p.obs_step_stride = (long long)c.n_envs * c.n_agents * c.obs_dim;
+  p.avail_step_stride = (long long)c.n_envs * c.n_agents * c.n_actions;
+  p.env_step_stride = c.n_envs;
+  p.actions_out = actions_out;
+  int rc;
+  if (a->use_tc) {
+    tc_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
+    rc = launch_actor_tc(p, a->sms, a->stream);
+  } else {
+    ffma_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
+    rc = launch_actor_ffma(p, a->sms, a->stream);
+  }
+  if (rc < 0) return fail(MARL_ECUDA, "actor kernel launch: %s", cudaGetErrorString((cudaError_t)(-rc)));
+  a->launches += (uint64_t)rc;
+  a->step += (uint64_t)T;
+  if (a->trace_actions || a->trace_q) {
+    const long long nx = (long long)a->trace_next + T;
+    a->trace_next = nx > a->trace_cap ? a->trace_cap : (int32_t)nx;
+  }
+  return MARL_OK;
+}
+
+int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                    const uint8_t* done, float eps, int32_t* actions_out) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
+  if (!(eps >= 0.0f && eps <= 1.0f)) return fail(MARL_EINVAL, "eps must be in [0, 1]");
+  return enqueue_steps(a, obs, avail, reward, done, 1, true, eps, 0, 0, 0, actions_out);
+}
+
+int marl_actor_step_host(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                         const uint8_t* done, float eps, int32_t* actions_out) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
+  if (!(eps >= 0.0f && eps <= 1.0f)) return fail(MARL_EINVAL, "eps must be in [0, 1]");
+  const marl_actor_config_t& c = a->cfg;
+  const WorkOffsets wo = work_offsets(c, 1);
+  const size_t rows = (size_t)c.n_envs * c.n_agents;
+  float* d_obs = reinterpret_cast<float*>(a->work + wo.obs);
+  uint8_t* d_avail = a->work + wo.avail;
+  float* d_reward = reinterpret_cast<float*>(a->work + wo.reward);
+  uint8_t* d_done = a->work + wo.done;
+  int32_t* d_act = reinterpret_cast<int32_t*>(a->work + wo.actions);
+  CU_TRY(cudaMemcpyAsync(d_obs, obs, sizeof(float) * rows * c.obs_dim, cudaMemcpyHostToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(d_avail, avail, rows * c.n_actions, cudaMemcpyHostToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(d_reward, reward, sizeof(float) * c.n_envs, cudaMemcpyHostToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(d_done, done, (size_t)c.n_envs, cudaMemcpyHostToDevice, a->stream));
+  const int rc = enqueue_steps(a, d_obs, d_avail, d_reward, d_done, 1, true, eps, 0, 0, 0, d_act);
+  if (rc) return rc;
+  if (actions_out)
+    CU_TRY(cudaMemcpyAsync(actions_out, d_act, sizeof(int32_t) * rows, cudaMemcpyDeviceToHost, a->stream));
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  return MARL_OK;
+}
+
+int marl_env_generate(const marl_actor_t* a_, const marl_synth_env_t* env, uint32_t t0, int32_t n_steps,
+                      float* obs, uint8_t* avail, float* reward, uint8_t* done) {
+  marl_actor* a = const_cast<marl_actor*>(a_);
+  if (!a || !env) return fail(MARL_EINVAL, "actor or env is NULL");
+  if (n_steps < 1) return fail(MARL_EINVAL, "n_steps must be >= 1");
+  if (!obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an output pointer is NULL");
+  if ((reinterpret_cast<uintptr_t>(obs) | reinterpret_cast<uintptr_t>(avail) | reinterpret_cast<uintptr_t>(reward) |
+       reinterpret_cast<uintptr_t>(done)) % 16)
+    return fail(MARL_EALIGN, "environment arrays must be 16-byte aligned");
+  if (env->obs_law != 0 && env->obs_law != 1) return fail(MARL_EINVAL, "obs_law must be 0 or 1");
+  if (env->obs_law == 1 && 2 * a->cfg.obs_dim + 1 >= 65536) return fail(MARL_EINVAL, "obs_dim too large for law 1");
+  const marl_actor_config_t& c = a->cfg;
+  const int rc = launch_env_generate(*env, c.n_envs, c.n_agents, c.obs_dim, c.n_actions, t0, n_steps, obs, avail,
+                                     reward, done, a->sms, a->stream);
+  if (rc < 0) return fail(MARL_ECUDA, "environment kernel launch: %s", cudaGetErrorString((cudaError_t)(-rc)));
+  a->launches += (uint64_t)rc;
+  return MARL_OK;
+}
+
+int marl_rollout_staged(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
+                        const uint8_t* done, int32_t T, double eps_start, double eps_end, int32_t anneal_steps) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
+  if (T < 1) return fail(MARL_EINVAL, "T must be >= 1");
+  if (!(eps_start >= 0.0 && eps_start <= 1.0 && eps_end >= 0.0 && eps_end <= 1.0))
+    return fail(MARL_EINVAL, "eps must be in [0, 1]");
+  return enqueue_steps(a, obs, avail, reward, done, T, false, 0.f, eps_start, eps_end, anneal_steps, nullptr);
+}
+
+int marl_rollout(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double eps_start, double eps_end,
+                 int32_t anneal_steps) {
+  if (!a || !env) return fail(MARL_EINVAL, "actor or env is NULL");
+  if (T < 1) return fail(MARL_EINVAL, "T must be >= 1");
+  const marl_actor_config_t& c = a->cfg;
+  // Largest window of steps whose staging fits the work buffer.
+  size_t W = 1;
+  while (W < (size_t)T && work_offsets(c, W + 1).total <= a->work_bytes) {
+    size_t W2 = W * 2 < (size_t)T ? W * 2 : (size_t)T;
+    if (work_offsets(c, W2).total <= a->work_bytes) W = W2; else W += 1;
+  }
+  const WorkOffsets wo = work_offsets(c, W);
+  float* d_obs = reinterpret_cast<float*>(a->work + wo.obs);
+  uint8_t* d_avail = a->work + wo.avail;
+  float* d_reward = reinterpret_cast<float*>(a->work + wo.reward);
+  uint8_t* d_done = a->work + wo.done;
+  int32_t left = T;
+  while (left > 0) {
+    const int32_t w = left < (int32_t)W ? left : (int32_t)W;
+    int rc = marl_env_generate(a, env, (uint32_t)a->step, w, d_obs, d_avail, d_reward, d_done);
+    if (rc) return rc;
+    rc = marl_rollout_staged(a, d_obs, d_avail, d_reward, d_done, w, eps_start, eps_end, anneal_steps);
+    if (rc) return rc;
+    left -= w;
+  }
+  return MARL_OK;
+}
+
+int marl_actor_set_trace(marl_actor_t* a, int32_t* actions, float* q, int32_t capacity_steps) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (capacity_steps < 0) return fail(MARL_EINVAL, "capacity_steps must be >= 0");
+  a->trace_actions = capacity_steps ? actions : nullptr;
+  a->trace_q = capacity_steps ? q : nullptr;
+  a->trace_cap = capacity_steps;
+  a->trace_next = 0;
+  return MARL_OK;
+}
+
+int marl_ring_view(const marl_actor_t* a, marl_ring_view_t* out) {
+  if (!a || !out) return fail(MARL_EINVAL, "actor or out is NULL");
+  const marl_actor_config_t& c = a->cfg;
+  out->base = a->ring + a->ro.records;
+  out->step_stride = a->rl.rec_bytes;
+  out->slot_stride = (size_t)c.ring_steps * a->rl.rec_bytes;
+  out->off_obs = a->rl.off_obs;
+  out->off_avail = a->rl.off_avail;
+  out->off_action = a->rl.off_action;
+  out->off_q = a->rl.off_q;
+  out->off_reward = a->rl.off_reward;
+  out->off_done = a->rl.off_done;
+  out->episodes = c.ring_episodes;
+  out->steps = c.ring_steps;
+  out->slots_per_env = c.ring_episodes / c.n_envs;
+  out->n_envs = c.n_envs;
+  out->n_agents = c.n_agents;
+  out->obs_dim = c.obs_dim;
+  out->n_actions = c.n_actions;
+  out->reserved = 0;
+  out->slot_epid = reinterpret_cast<int64_t*>(a->ring + a->ro.epid);
+  out->slot_len = reinterpret_cast<int32_t*>(a->ring + a->ro.len);
+  out->slot_complete = a->ring + a->ro.complete;
+  return MARL_OK;
+}
+
+int marl_actor_get_state(const marl_actor_t* a, marl_state_view_t* out) {
+  if (!a || !out) return fail(MARL_EINVAL, "actor or out is NULL");
+  uint8_t* st = a->state;
+  out->h = reinterpret_cast<float*>(st + a->so.h);
+  out->last_action = reinterpret_cast<int32_t*>(st + a->so.last_action);
+  out->slot = reinterpret_cast<int32_t*>(st + a->so.slot);
+  out->pos = reinterpret_cast<int32_t*>(st + a->so.pos);
+  out->ep_count = reinterpret_cast<int64_t*>(st + a->so.ep_count);
+  out->step = a->step;
+  return MARL_OK;
+}
+
+int marl_actor_set_state(marl_actor_t* a, const marl_state_view_t* in) {
+  if (!a || !in) return fail(MARL_EINVAL, "actor or in is NULL");
+  if (!in->h || !in->last_action || !in->slot || !in->pos || !in->ep_count) return fail(MARL_EINVAL, "a state pointer is NULL");
+  if (in->step > 0xFFFFFFFFull) return fail(MARL_EINVAL, "step counter exceeds 32 bits");
+  const marl_actor_config_t& c = a->cfg;
+  const size_t rows = (size_t)c.n_envs * c.n_agents;
+  uint8_t* st = a->state;
+  CU_TRY(cudaMemcpyAsync(st + a->so.h, in->h, sizeof(float) * rows * c.hidden, cudaMemcpyDeviceToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(st + a->so.last_action, in->last_action, sizeof(int32_t) * rows, cudaMemcpyDeviceToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(st + a->so.slot, in->slot, sizeof(int32_t) * c.n_envs, cudaMemcpyDeviceToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(st + a->so.pos, in->pos, sizeof(int32_t) * c.n_envs, cudaMemcpyDeviceToDevice, a->stream));
+  CU_TRY(cudaMemcpyAsync(st + a->so.ep_count, in->ep_count, sizeof(int64_t) * c.n_envs, cudaMemcpyDeviceToDevice, a->stream));
+  a->step = in->step;
+  return MARL_OK;
+}
+
+int marl_actor_status(marl_actor_t* a, uint32_t* device_status, marl_counters_t* counters) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  uint64_t cnt[CNT_N];
+  uint32_t st = 0;
+  CU_TRY(cudaMemcpyAsync(cnt, a->state + a->so.counters, sizeof(cnt), cudaMemcpyDeviceToHost, a->stream));
+  CU_TRY(cudaMemcpyAsync(&st, a->state + a->so.status, sizeof(st), cudaMemcpyDeviceToHost, a->stream));
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  if (device_status) *device_status = st;
+  if (counters) {
+    counters->agent_steps = cnt[CNT_AGENT_STEPS];
+    counters->episodes = cnt[CNT_EPISODES];
+    counters->explored = cnt[CNT_EXPLORED];
+    counters->no_avail = cnt[CNT_NO_AVAIL];
+    counters->truncated = cnt[CNT_TRUNCATED];
+  }
+  return MARL_OK;
+}
+
+int marl_actor_reset(marl_actor_t* a) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  return enqueue_reset(a);
+}
+
+const char* marl_actor_kernel_name(const marl_actor_t* a) { return (a && a->use_tc) ? "tcgen05" : "ffma"; }
+
+uint64_t marl_actor_launch_count(const marl_actor_t* a) { return a ? a->launches : 0; }
+
+}  // extern "C"

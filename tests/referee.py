@@ -1,0 +1,139 @@
+"""Parity referee: compares a rollout of the CUDA library with the CPU oracle.
+
+A double-precision CPU loop and a GPU kernel cannot agree on every near-tie of the greedy rule, and one
+differing action changes the rest of that environment's trajectory (the action is fed back as an input).
+So parity is split into parts that are each decidable:
+
+1. integer-derived quantities (environment streams, done flags, ring cursors and headers, counters): exact;
+2. the decision given Q: the oracle's selection applied to the GPU's own stored Q row, the mask and the
+   Philox draw must reproduce the GPU's action exactly, for every row;
+3. values: Q and hidden state within the relative tolerance (row-wise infinity norm, floor 1e-3);
+4. free-running agreement: where the oracle's own choice differs from the GPU's although 2 and 3 hold,
+   the row is a numerical near-tie; it is counted, and the oracle adopts the GPU's action so that both stay
+   in lock-step.  The count must stay under a stated budget.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2205_05248_b200 import binding, workloads
+
+RTOL = {"fp32": 1e-5, "bf16": 2e-2}
+
+
+def row_rel_err(got: np.ndarray, want: np.ndarray) -> np.ndarray:
+    """max|got-want| / max(max|want|, 1e-3) over the last axis."""
+    num = np.max(np.abs(got.astype(np.float64) - want.astype(np.float64)), axis=-1)
+    den = np.maximum(np.max(np.abs(want.astype(np.float64)), axis=-1), 1e-3)
+    return num / den
+
+
+def eps_schedule(cfg, t0, T):
+    return np.array([oracle.eps_at(cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], t0 + k)
+                     for k in range(T)], np.float32)
+
+
+def run_gpu_rollout(cfg, weights, kernel="auto", T=None, splits=None, want_q=True, work_steps=None):
+    """Runs marl_rollout (optionally as several consecutive calls) with the trace on.  Returns the actor and
+    the traced actions / Q as device tensors."""
+    T = cfg["T"] if T is None else T
+    actor = binding.Actor(cfg, kernel=kernel, work_steps=work_steps)
+    actor.set_weights(weights)
+    acts, q = actor.set_trace(T, want_q=want_q)
+    for part in (splits or [T]):
+        actor.rollout(cfg["env"], part, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+    torch.cuda.synchronize()
+    return actor, acts, q
+
+
+def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=1e-4, n_threads=None):
+    """Checks parts 1-4 for the listed environments (default: all).  Returns a summary dict."""
+    T = cfg["T"] if T is None else T
+    E, n, A, H = cfg["E"], cfg["n"], cfg["A"], cfg["H"]
+    ids = np.arange(E) if env_ids is None else np.asarray(env_ids)
+    rtol = RTOL[cfg["precision"]]
+    tids = torch.as_tensor(ids, device=gpu_actions.device, dtype=torch.long)
+    g_act = gpu_actions[:T].index_select(1, tids).cpu().numpy()
+    g_q = gpu_q[:T].index_select(1, tids).cpu().numpy()
+
+    sess = oracle.Session(cfg, weights, ids, n_threads=n_threads or oracle.hardware_threads())
+    tr = sess.rollout(cfg["env"], T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], adopt=g_act)
+
+    # ---- part 2: the GPU's decision follows from its own Q row ----
+    eps = eps_schedule(cfg, 0, T)
+    N = T * len(ids) * n
+    tt = np.repeat(np.arange(T, dtype=np.uint32), len(ids) * n)
+    ee = np.tile(np.repeat(ids.astype(np.uint32), n), T)
+    ii = np.tile(np.arange(n, dtype=np.uint32), T * len(ids))
+    re_act, re_ex = oracle.select_batch(g_q.reshape(N, A), tr["avail"].reshape(N, A), eps[tt], cfg["seed"], tt, ee, ii)
+    bad = np.nonzero(re_act != g_act.reshape(N))[0]
+    assert bad.size == 0, f"decision-given-Q mismatch at rows {bad[:8]} (t,e,i)={[(tt[b], ee[b], ii[b]) for b in bad[:4]]}"
+    assert np.array_equal(re_ex, tr["explore"].reshape(N)), "explore flags differ"
+    assert np.take_along_axis(tr["avail"], g_act[..., None].astype(np.int64), axis=-1).all(), "unavailable action chosen"
+
+    # ---- part 3: values ----
+    q_err = row_rel_err(g_q, tr["q"])
+    assert q_err.max() <= rtol, f"Q error {q_err.max():.3e} > {rtol} at {np.unravel_index(q_err.argmax(), q_err.shape)}"
+    st = actor.get_state()
+    g_h = st["h"].index_select(0, tids).cpu().numpy()
+    h_err = row_rel_err(g_h, sess.h)
+    assert h_err.max() <= rtol, f"final h error {h_err.max():.3e} > {rtol}"
+
+    # ---- part 4: near-ties ----
+    greedy_rows = int((tr["explore"] == 0).sum())
+    near = np.argwhere(tr["action_free"] != g_act)
+    for (t, x, i) in near[:64]:
+        assert tr["explore"][t, x, i] == 0
+        a_o, a_g = tr["action_free"][t, x, i], g_act[t, x, i]
+        gap = abs(float(tr["q"][t, x, i, a_o]) - float(tr["q"][t, x, i, a_g]))
+        scale = max(float(np.max(np.abs(tr["q"][t, x, i]))), 1e-3)
+        assert gap <= 1e-4 + 2 * rtol * scale, f"actions differ at {(t, x, i)} with an oracle Q gap of {gap:.3e}"
+    frac = len(near) / max(greedy_rows, 1)
+    assert frac <= near_tie_budget, f"{len(near)} near-ties in {greedy_rows} greedy decisions"
+
+    # ---- part 1: integer state, ring and headers ----
+    assert np.array_equal(st["last_action"].index_select(0, tids).cpu().numpy(), sess.last_action)
+    assert np.array_equal(st["slot"].index_select(0, tids).cpu().numpy(), sess.slot)
+    assert np.array_equal(st["pos"].index_select(0, tids).cpu().numpy(), sess.pos)
+    assert np.array_equal(st["ep_count"].index_select(0, tids).cpu().numpy(), sess.ep_count)
+    assert st["step"] == T
+    rv = actor.ring_view()
+    S = sess.S
+    slots = (ids[:, None] * S + np.arange(S)[None, :]).reshape(-1)
+    tsl = torch.as_tensor(slots, device=gpu_actions.device, dtype=torch.long)
+    hdr_len = rv["slot_len"].index_select(0, tsl).cpu().numpy()
+    assert np.array_equal(rv["slot_epid"].index_select(0, tsl).cpu().numpy(), sess.ring["slot_epid"])
+    assert np.array_equal(hdr_len, sess.ring["slot_len"])
+    assert np.array_equal(rv["slot_complete"].index_select(0, tsl).cpu().numpy(), sess.ring["slot_complete"])
+    # rows that have been written (per slot: the first max-written positions); compare only those
+    written = np.zeros((len(slots), cfg["L"]), bool)
+    for t in range(T):
+        loc = tr["slot"][t] - ids * S + np.arange(len(ids)) * S
+        written[loc, tr["pos"][t]] = True
+    for name in ("obs", "avail", "action", "reward", "done"):
+        g = rv[name].index_select(0, tsl).cpu().numpy()
+        assert np.array_equal(g[written], sess.ring[name][written]), f"ring field {name} differs"
+    gq = rv["q"].index_select(0, tsl).cpu().numpy()
+    rq_err = row_rel_err(gq[written], sess.ring["q"][written])
+    assert rq_err.max() <= rtol, f"ring Q error {rq_err.max():.3e}"
+
+    status, counters = actor.status()
+    assert status == 0, f"device status {status}"
+    if len(ids) == E:
+        oc = sess.counters
+        assert counters["agent_steps"] == oc[oracle.CNT_STEPS] and counters["episodes"] == oc[oracle.CNT_EPISODES]
+        assert counters["explored"] == oc[oracle.CNT_EXPLORE] and counters["truncated"] == oc[oracle.CNT_TRUNCATED]
+        assert counters["no_avail"] == oc[oracle.CNT_NO_AVAIL]
+    return dict(near_ties=len(near), greedy_rows=greedy_rows, q_err=float(q_err.max()), h_err=float(h_err.max()),
+                rows=N, episodes=int(sess.counters[oracle.CNT_EPISODES]), kernel=actor.kernel_name)
+
+
+def sample_envs(E: int, count: int, seed: int = 0) -> np.ndarray:
+    """A seeded subset of environment ids that always contains the first and the last."""
+    if count >= E:
+        return np.arange(E)
+    rng = np.random.default_rng(seed)
+    ids = set(rng.choice(E, size=count, replace=False).tolist()) | {0, E - 1}
+    return np.array(sorted(ids))

@@ -1,0 +1,230 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2205_05248_b200 import binding, workloads
+from referee import RTOL, referee, row_rel_err, run_gpu_rollout, sample_envs
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_env_block(cfg, ids, t0, n_steps):
+    obs = np.zeros((n_steps, len(ids), cfg["n"], cfg["D"]), np.float32)
+    avail = np.zeros((n_steps, len(ids), cfg["n"], cfg["A"]), np.uint8)
+    rew = np.zeros((n_steps, len(ids)), np.float32)
+    done = np.zeros((n_steps, len(ids)), np.uint8)
+    for s in range(n_steps):
+        for x, e in enumerate(ids):
+            obs[s, x], avail[s, x], rew[s, x], done[s, x] = oracle.env_emit(cfg, cfg["env"], t0 + s, int(e))
+    return obs, avail, rew, done
+
+
+@pytest.mark.parametrize("k,t0,n_steps,n_ids", [(1, 0, 16, 8), (2, 5, 3, 24), (3, 250, 2, 24), (4, 77, 2, 24),
+                                                (5, 63, 1, 16)])
+def test_env_generate_bit_exact(k, t0, n_steps, n_ids):
+    """Every synthetic-environment stream equals the oracle's, bit for bit, at the full batch size."""
+    cfg = workloads.config(k, E=4096) if k == 5 else workloads.config(k)
+    actor = binding.Actor(cfg, kernel="ffma", work_steps=1)
+    obs, avail, rew, done = actor.env_generate(cfg["env"], t0, n_steps)
+    ids = sample_envs(cfg["E"], n_ids, seed=k)
+    t = torch.as_tensor(ids, device=obs.device)
+    o_obs, o_avail, o_rew, o_done = _oracle_env_block(cfg, ids, t0, n_steps)
+    assert np.array_equal(obs.index_select(1, t).cpu().numpy().view(np.uint32), o_obs.view(np.uint32))
+    assert np.array_equal(avail.index_select(1, t).cpu().numpy(), o_avail)
+    assert np.array_equal(rew.index_select(1, t).cpu().numpy().view(np.uint32), o_rew.view(np.uint32))
+    assert np.array_equal(done.index_select(1, t).cpu().numpy(), o_done)
+    # whole-batch properties that hold at any size
+    assert bool((avail[..., 0] == 1).all())
+    assert float(obs.abs().max()) <= 3.0
+    actor.destroy()
+
+
+def test_config1_full_parity_fp32():
+    """Workload 1 (3 agents, fp32): every row of every step, no near-tie allowed."""
+    cfg = workloads.config(1)
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w)
+    res = referee(cfg, w, actor, acts, q, near_tie_budget=0.0)
+    assert res["rows"] == 384 and res["kernel"] == "ffma"
+    actor.destroy()
+
+
+@pytest.mark.parametrize("k,n_ids", [(2, 160), (3, 96), (4, 160)])
+def test_configs_2_to_4_parity(k, n_ids):
+    """Full-size GPU rollout; the oracle recomputes a seeded subset of environments in isolation."""
+    cfg = workloads.config(k)
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w)
+    ids = sample_envs(cfg["E"], n_ids, seed=k)
+    res = referee(cfg, w, actor, acts, q, env_ids=ids)
+    print(f"cfg{k}: {res}")
+    # properties over the whole batch: every chosen action is available; every step was recorded
+    rv = actor.ring_view()
+    status, counters = actor.status()
+    assert status == 0 and counters["agent_steps"] == cfg["E"] * cfg["n"] * cfg["T"]
+    lens = rv["slot_len"].cpu().numpy()
+    assert lens.max() <= cfg["L"]
+    actor.destroy()
+
+
+@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "ffma"), (128, "bf16", "ffma"), (64, "fp32", "ffma"),
+                                           (128, "fp32", "ffma")])
+def test_config5_parity_small_E(H, prec, kernel):
+    cfg = workloads.config(5, E=4096, H=H, precision=prec)
+    cfg["T"] = 24
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
+    res = referee(cfg, w, actor, acts, q, env_ids=sample_envs(cfg["E"], 48, seed=H))
+    print(f"cfg5 H={H} {prec}: {res}")
+    actor.destroy()
+
+
+def test_ragged_tiles_and_tiny_shapes():
+    """Tile tails (E not a multiple of the tile), one agent, one action, one environment."""
+    for over in (dict(E=37, n=5, C=74), dict(E=1, n=1, A=1, C=2), dict(E=150, n=7, A=32, D=3, C=150),
+                 dict(E=9, n=32, A=2, D=17, C=9), dict(E=300, n=3, D=129, C=300)):
+        cfg = workloads.small_config(H=64, L=7, T=20, **over)
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="ffma")
+        referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
+        actor.destroy()
+
+
+def test_done_every_step_and_never():
+    for thr, L in ((1 << 24, 4), (0, 5)):
+        cfg = workloads.small_config(H=64, E=40, C=80, L=L, T=17, env=dict(done_thresh24=thr))
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="ffma")
+        res = referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
+        _, counters = actor.status()
+        if thr:
+            assert counters["episodes"] == 40 * 17 and counters["truncated"] == 0
+        else:
+            assert counters["truncated"] == counters["episodes"] == 40 * (17 // 5)
+        actor.destroy()
+
+
+def test_annealed_epsilon_and_split_rollouts_resume():
+    """eps schedule follows the global step; rollout(T) == rollout(a) + rollout(b); a checkpoint restored
+    into a fresh handle continues identically."""
+    cfg = workloads.small_config(H=64, E=64, C=128, L=9, T=30, eps_start=1.0, eps_end=0.05, anneal_steps=29)
+    w = workloads.make_weights(cfg)
+    one, a1, q1 = run_gpu_rollout(cfg, w, kernel="ffma")
+    referee(cfg, w, one, a1, q1, near_tie_budget=2e-3)
+    two, a2, q2 = run_gpu_rollout(cfg, w, kernel="ffma", splits=[11, 19])
+    assert torch.equal(a1, a2) and torch.equal(q1, q2)
+    r1, r2 = one.ring_view(), two.ring_view()
+    assert torch.equal(one.ring_mem, two.ring_mem)
+    # checkpoint after 11 steps -> fresh handle -> 19 more
+    first = binding.Actor(cfg, kernel="ffma")
+    first.set_weights(w)
+    first.rollout(cfg["env"], 11, 1.0, 0.05, 29)
+    st = first.get_state()
+    second = binding.Actor(cfg, kernel="ffma")
+    second.set_weights(w)
+    second.ring_mem.copy_(first.ring_mem)
+    second.set_state(st)
+    second.rollout(cfg["env"], 19, 1.0, 0.05, 29)
+    torch.cuda.synchronize()
+    assert torch.equal(second.ring_mem, one.ring_mem)
+    s1, s2 = one.get_state(), second.get_state()
+    for key in ("h", "last_action", "slot", "pos", "ep_count"):
+        assert torch.equal(s1[key], s2[key]), key
+    assert s1["step"] == s2["step"] == 30
+    for a in (one, two, first, second):
+        a.destroy()
+
+
+def test_step_api_equals_rollout_and_host_variant():
+    """T calls of marl_actor_step (device inputs) and of marl_actor_step_host (host inputs) reproduce
+    marl_rollout: same actions, same ring, same state."""
+    cfg = workloads.small_config(H=64, E=50, n=4, C=100, L=8, T=12)
+    w = workloads.make_weights(cfg)
+    ref, acts, q = run_gpu_rollout(cfg, w, kernel="ffma")
+    obs, avail, rew, done = ref.env_generate(cfg["env"], 0, cfg["T"])
+    dev = binding.Actor(cfg, kernel="ffma")
+    dev.set_weights(w)
+    host = binding.Actor(cfg, kernel="ffma")
+    host.set_weights(w)
+    h_obs, h_avail, h_rew, h_done = [t.cpu().pin_memory() for t in (obs, avail, rew, done)]
+    h_act = torch.empty((cfg["E"], cfg["n"]), dtype=torch.int32).pin_memory()
+    for t in range(cfg["T"]):
+        a = dev.step(obs[t], avail[t], rew[t], done[t], cfg["eps_start"])
+        assert torch.equal(a, acts[t])
+        host.step_host(h_obs[t], h_avail[t], h_rew[t], h_done[t], cfg["eps_start"], h_act)
+        assert torch.equal(h_act, acts[t].cpu())
+    torch.cuda.synchronize()
+    assert torch.equal(dev.ring_mem, ref.ring_mem) and torch.equal(host.ring_mem, ref.ring_mem)
+    for key in ("h", "last_action", "slot", "pos", "ep_count"):
+        assert torch.equal(dev.get_state()[key], ref.get_state()[key]), key
+    for a in (ref, dev, host):
+        a.destroy()
+
+
+def test_determinism_same_seed_same_bytes():
+    cfg = workloads.config(2, E=512)
+    cfg["T"] = 16
+    w = workloads.make_weights(cfg)
+    a, acts_a, q_a = run_gpu_rollout(cfg, w)
+    b, acts_b, q_b = run_gpu_rollout(cfg, w)
+    assert torch.equal(acts_a, acts_b) and torch.equal(q_a, q_b)
+    ra, rb = a.ring_view(), b.ring_view()
+    for k in ("obs", "avail", "action", "q", "reward", "done", "slot_epid", "slot_len", "slot_complete"):
+        assert torch.equal(ra[k], rb[k]), k
+    a.destroy()
+    b.destroy()
+
+
+def test_no_available_action_is_reported_not_fatal():
+    """A row whose mask is all zero takes action 0, sets the status bit and counts it."""
+    cfg = workloads.small_config(H=64, E=6, n=2, C=6, L=8, T=1)
+    w = workloads.make_weights(cfg)
+    actor = binding.Actor(cfg, kernel="ffma")
+    actor.set_weights(w)
+    obs, avail, rew, done = actor.env_generate(cfg["env"], 0, 1)
+    avail[0, 3, 1, :] = 0
+    acts = actor.step(obs[0], avail[0], rew[0], done[0], 0.0)
+    status, counters = actor.status()
+    assert status & binding.STATUS_NO_AVAIL and counters["no_avail"] == 1
+    assert int(acts[3, 1]) == 0
+    sess = oracle.Session(cfg, w, np.arange(cfg["E"]))
+    o_acts, _ = sess.step(obs[0].cpu().numpy(), avail[0].cpu().numpy(), rew[0].cpu().numpy(), done[0].cpu().numpy(), 0.0)
+    assert np.array_equal(acts.cpu().numpy(), o_acts) and sess.counters[oracle.CNT_NO_AVAIL] == 1
+    actor.destroy()
+
+
+def test_bad_cursor_sets_status_and_skips():
+    """A corrupted ring cursor handed in through set_state is detected; nothing is written out of range."""
+    cfg = workloads.small_config(H=64, E=4, C=4, L=8, T=2)
+    w = workloads.make_weights(cfg)
+    actor = binding.Actor(cfg, kernel="ffma")
+    actor.set_weights(w)
+    st = actor.get_state()
+    bad = {k: (v.clone() if torch.is_tensor(v) else v) for k, v in st.items()}
+    bad["pos"][2] = 99
+    actor.set_state(bad)
+    before = actor.ring_mem.clone()
+    actor.rollout(cfg["env"], 2, 0.1)
+    status, _ = actor.status()
+    assert status & binding.STATUS_BAD_INDEX
+    rv = actor.ring_view()
+    assert int(rv["slot_len"][2]) == 0
+    actor.destroy()
+
+
+def test_host_errors_are_codes_not_crashes():
+    cfg = workloads.small_config(H=64)
+    actor = binding.Actor(cfg, kernel="ffma")
+    obs, avail, rew, done = actor.env_generate(cfg["env"], 0, 1)
+    with pytest.raises(binding.MarlError, match="set_weights"):
+        actor.step(obs[0], avail[0], rew[0], done[0], 0.1)
+    actor.set_weights(workloads.make_weights(cfg))
+    with pytest.raises(binding.MarlError, match="eps"):
+        actor.step(obs[0], avail[0], rew[0], done[0], 1.5)
+    with pytest.raises(binding.MarlError):
+        actor.rollout(cfg["env"], 0, 0.1)
+    actor.destroy()
+    with pytest.raises(binding.MarlError, match="tensor-core"):
+        binding.Actor(dict(cfg, precision="fp32"), kernel="tensor")
