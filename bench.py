@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the batched actor path: agent-steps per second on one B200, ring write included.
+
+One bench "step" is one ``marl_rollout_staged`` call: T environment steps over all E environments, i.e. one
+pass of the whole hot path (stage obs, network, choice, ring write, episode bookkeeping) over one batch of
+synthetic environment output that is already resident in HBM (generated once, before the timed region,
+by ``marl_env_generate``).  The default workload is the largest one of the throughput sweep
+(E=65536 x 8 agents, obs 80, 14 actions, hidden 64, bf16, T=64, ring of about 20 GB).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 5 --E 65536 --H 64 --precision bf16]
+                    [--kernel auto|ffma|tensor] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torchrun, one rank per GPU) every rank runs its own
+replica of the workload - environments are independent, there is no data-path collective - and the value
+is the sum over ranks divided by the slowest rank's time ("weak" scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+METRIC = "agent-steps/sec at 1 B200 (incl. ring write); % of step roofline (HBM/TC)"
+UNIT = "agent-steps/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=5)
+    ap.add_argument("--E", type=int, default=None)
+    ap.add_argument("--H", type=int, default=None)
+    ap.add_argument("--precision", default=None, choices=[None, "fp32", "bf16"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def algorithmic_bytes_per_agent_step(cfg: dict, T: int) -> float:
+    """Bytes that one agent-step of a tile-major rollout must move to and from HBM:
+    reads  obs 4D + avail A + (reward 4 + done 1)/n, writes the ring record's payload
+    obs 4D + avail A + action 4 + Q 4A + (reward 4 + done 1)/n, plus the hidden state loaded and stored once
+    per launch (8H/T).  Padding, headers and weights are not counted."""
+    D, A, n, H = cfg["D"], cfg["A"], cfg["n"], cfg["H"]
+    reads = 4 * D + A + 5.0 / n
+    writes = 4 * D + A + 4 + 4 * A + 5.0 / n
+    return reads + writes + 8.0 * H / T
+
+
+def flops_per_agent_step(cfg: dict) -> float:
+    D, A, H = cfg["D"], cfg["A"], cfg["H"]
+    return 2.0 * H * (D + 6 * H + A) + 25.0 * H
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        inside = [r for (ts, r) in self.rows if t_begin <= ts <= t_end + 0.05] or [r for (_, r) in self.rows]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in inside:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    """Returns (rank, world, local_rank).  torch.distributed is used only for the barrier and the max of the
+    per-rank times; the data path has no collective."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return rank, world, local
+
+
+def dist_max(value: float, world: int, device="cuda") -> float:
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def dist_barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def cpu_baseline(cfg: dict, weights: dict, budget_s: float = 15.0) -> dict:
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    import numpy as np
+    import oracle
+    cores = oracle.hardware_threads()
+    T = cfg["T"]
+    probe = min(cfg["E"], max(cores, 8))
+    sess = oracle.Session(cfg, weights, np.arange(probe), with_ring=True, n_threads=cores)
+    t0 = time.perf_counter()
+    sess.rollout(cfg["env"], min(T, 8), cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], trace=())
+    dt = time.perf_counter() - t0
+    rate = probe * cfg["n"] * min(T, 8) / dt
+    envs = int(min(cfg["E"], max(probe, rate * budget_s / (cfg["n"] * T))))
+    sess = oracle.Session(cfg, weights, np.arange(envs), with_ring=True, n_threads=cores)
+    t0 = time.perf_counter()
+    sess.rollout(cfg["env"], T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], trace=())
+    dt = time.perf_counter() - t0
+    return {"value": envs * cfg["n"] * T / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {envs} of {cfg['E']} environments x T={T} steps, {dt:.1f} s"}
+
+
+def run_reference(args, cfg, rank):
+    """--impl reference: the CPU oracle on the host cores, same metric and workload, bounded sample per step."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2205_05248_b200 import workloads
+    weights = workloads.make_weights(cfg)
+    cores = oracle.hardware_threads()
+    T = cfg["T"]
+    envs = min(cfg["E"], 4 * cores)
+    times = []
+    for k in range(args.warmup + args.steps):
+        sess = oracle.Session(cfg, weights, np.arange(envs), with_ring=True, n_threads=cores)
+        t0 = time.perf_counter()
+        sess.rollout(cfg["env"], T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], trace=())
+        dt = time.perf_counter() - t0
+        if k >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = envs * cfg["n"] * T * len(times) / total
+    sample = f"first {envs} of {cfg['E']} environments x T={T} steps per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg["name"], "step": f"one rollout of T={T} steps", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    from paper_2205_05248_b200 import workloads
+    cfg = workloads.config(args.workload, E=args.E, H=args.H, precision=args.precision)
+    rank, world, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    from paper_2205_05248_b200 import binding
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    cfg["seed"] = cfg["seed"] + (rank << 20)          # every rank runs its own replica
+    cfg["env"] = dict(cfg["env"], seed=cfg["env"]["seed"] + (rank << 20))
+    T, E, n = cfg["T"], cfg["E"], cfg["n"]
+    weights = workloads.make_weights(cfg)
+
+    actor = binding.Actor(cfg, device=str(dev), kernel=args.kernel, work_steps=1)
+    actor.set_weights(weights)
+    staged = actor.env_generate(cfg["env"], 0, T)      # resident in HBM before the timed region
+    input_bytes = sum(t.numel() * t.element_size() for t in staged)
+    torch.cuda.synchronize()
+
+    def one_step():
+        actor.rollout_staged(*staged, T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize()
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = actor.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist_barrier(world)
+    torch.cuda.synchronize()
+    t_begin = time.perf_counter()
+    ev0.record()
+    for _ in range(args.steps):
+        one_step()
+    ev1.record()
+    torch.cuda.synchronize()
+    t_end = time.perf_counter()
+    dist_barrier(world)
+    clocks = sampler.stop(t_begin, t_end)
+    launches = actor.launch_count - launches0
+    ms_local = ev0.elapsed_time(ev1)
+    ms_total = dist_max(ms_local, world)
+    status, counters = actor.status()
+    assert status == 0, f"device status {status}"
+    agent_steps = E * n * T * args.steps
+    value = world * agent_steps / (ms_total * 1e-3)
+
+    peaks, peak_kind = load_peaks()
+    kernel_ms = ms_local / max(launches, 1)            # one actor kernel per bench step
+    bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T) * E * n * T
+    achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
+    flop_rate = flops_per_agent_step(cfg) * E * n * T / (kernel_ms * 1e-3) / 1e12
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
+                "kernel": "actor_%s_kernel" % ("tc" if actor.kernel_name == "tcgen05" else "ffma"),
+                "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T),
+                "tflops_effective": flop_rate}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic",
+            "config": {"workload": cfg["name"], "E": E, "n": n, "D": cfg["D"], "A": cfg["A"], "H": cfg["H"], "T": T,
+                       "ring": f"{cfg['C']}x{cfg['L']}", "kernel": actor.kernel_name,
+                       "step": f"one marl_rollout_staged call = T={T} environment steps over E={E} environments",
+                       "l2": f"inputs larger than L2 ({input_bytes / 1e6:.0f} MB staged per step, read once)"},
+            "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline}
+
+    # ---- end to end through the host-buffer entry point: H2D of each step's inputs, D2H of its actions ----
+    if not args.no_e2e:
+        distinct = min(T, 4)
+        host = [[t[k].cpu().pin_memory() for t in staged] for k in range(distinct)]
+        h_act = torch.empty((E, n), dtype=torch.int32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in host[0]) * T
+        d2h = h_act.numel() * 4 * T
+        e2e_steps = max(1, min(args.steps, 5))
+        for k in range(2):
+            actor.step_host(*host[k % distinct], cfg["eps_start"], h_act)
+        dist_barrier(world)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for k in range(T):
+                actor.step_host(*host[k % distinct], cfg["eps_start"], h_act)
+        torch.cuda.synchronize()
+        dt = dist_max(time.perf_counter() - t0, world)
+        line["e2e"] = {"value": world * E * n * T * e2e_steps / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                       "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+                       "call": "marl_actor_step_host x T per step (pinned host buffers, actions read back)"}
+        del host
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        actor.destroy()
+        del staged
+        line["cpu_baseline"] = cpu_baseline(cfg, weights)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
