@@ -207,6 +207,26 @@ int marl_rollout_staged(marl_actor_t* a, const float* obs, const uint8_t* avail,
 int marl_rollout(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double eps_start, double eps_end,
                  int32_t anneal_steps);
 
+/* No counterpart in the paper: an integration variant of marl_rollout for callers that cannot allocate
+ * device memory - programs that gave all of it to their own pool at start-up, or that must avoid cudaMalloc
+ * because it synchronises the device and may fail in the middle of a run.  Same arguments and same results as
+ * marl_rollout, but the staging window for the generated environment steps is a fixed array of
+ * MARL_NOALLOC_SCRATCH_BYTES inside the library image instead of the actor's work buffer; the call performs
+ * no cudaMalloc, cudaFree or other allocating call.  (Create the actor on caller-provided ring, state and work
+ * buffers, otherwise marl_actor_create has already allocated.)
+ *   - every GPU that loads the library holds the array until the process exits;
+ *   - MARL_ENOMEM if one environment step of staging (E*n*(4D+A) + 5E bytes plus alignment) exceeds the
+ *     array; longer rollouts run in several windows;
+ *   - the array is shared by all actors and calls on a device and keeps the previous call's bytes; nothing
+ *     in it needs clearing, since each window is fully rewritten before it is read, but calls whose GPU work
+ *     overlaps race on it - serialise them;
+ *   - the first call on a device looks up the array's device address; make that call outside stream capture.
+ * The actor's device must be current, as for every other call.  Error text is not set for the size and
+ * look-up failures of this function itself; the return code tells them apart. */
+#define MARL_NOALLOC_SCRATCH_BYTES (32u << 20)
+int marl_rollout_noalloc(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double eps_start,
+                         double eps_end, int32_t anneal_steps);
+
 /* Optional per-step trace for verification: from the next step on, step k after this call writes its
  * actions to actions[k][E][n] and its Q rows to q[k][E][n][A] (device; either may be NULL) while
  * k < capacity_steps.  Pass NULL, NULL, 0 to switch it off. */

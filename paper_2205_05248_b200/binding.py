@@ -26,7 +26,7 @@ EXPORTS = [
     "marl_actor_step", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
     "marl_actor_set_trace", "marl_ring_view", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
-    "marl_actor_launch_count", "marl_last_error",
+    "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc",
 ]
 
 
@@ -102,6 +102,7 @@ def load_library():
         lib.marl_env_generate.argtypes = [P, C.POINTER(SynthEnv), C.c_uint32, C.c_int32, P, P, P, P]
         lib.marl_rollout_staged.argtypes = [P, P, P, P, P, C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
+        lib.marl_rollout_noalloc.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_actor_set_trace.argtypes = [P, P, P, C.c_int32]
         lib.marl_ring_view.argtypes = [P, C.POINTER(RingView)]
         lib.marl_actor_get_state.argtypes = [P, C.POINTER(StateView)]
@@ -246,6 +247,18 @@ class Actor:
         ev = make_env(env)
         _check(self.lib.marl_rollout(self.handle, C.byref(ev), C.c_int32(T), C.c_double(eps_start),
                                      C.c_double(eps_end), C.c_int32(anneal_steps)))
+
+    def rollout_noalloc(self, env: dict, T: int, eps_start: float, eps_end: float | None = None,
+                        anneal_steps: int = 0):
+        """marl_rollout_noalloc: same results as ``rollout``, staged through the library's fixed scratch array
+        (for callers that may not allocate device memory).  On failure the exception carries the return code, so
+        "too large for the scratch" (-4, MARL_ENOMEM) can be told from other errors."""
+        eps_end = eps_start if eps_end is None else eps_end
+        ev = make_env(env)
+        rc = self.lib.marl_rollout_noalloc(self.handle, C.byref(ev), C.c_int32(T), C.c_double(eps_start),
+                                           C.c_double(eps_end), C.c_int32(anneal_steps))
+        if rc != 0:
+            raise MarlError(f"marl_rollout_noalloc failed with code {rc}")
 
     # -- verification trace -----------------------------------------------------------------------
     def set_trace(self, capacity_steps: int, want_q: bool = True):
