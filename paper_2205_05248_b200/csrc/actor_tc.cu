@@ -1,12 +1,612 @@
-// Tensor-core (tcgen05) actor kernel - placeholder until the kernel lands: reports "unsupported" for
-// every shape, so the runtime always selects the FFMA kernel.
+// Tensor-core actor kernel for sm_100a: bf16 operands, hidden size 64, observation width a multiple of 8.
+//
+// Schedule (as in the FFMA kernel): one thread block owns a tile of whole environments - up to 128 agent
+// rows, the M of one tcgen05.mma - and runs all T steps of the launch for it before the next tile, because
+// environments never exchange data (Sec. III-A, Fig. 3).  Hidden state (fp32, in registers), last actions
+// and ring cursors stay on chip for the whole launch.
+//
+// Per step, the worker's decision (Algorithm 2) and the actor's recording (Algorithm 1) become:
+//   bulk-async load of the tile's observations, one copy per environment, straight into that environment's
+//   ring record being assembled in shared memory
+//   -> bf16 copy of the observations in the UMMA operand layout
+//   -> fc1 on the tensor core (accumulator in tensor memory) -> +bias, +one-hot columns, ReLU, bf16 (epilogue 1)
+//   -> the two GRU gate GEMMs (r|z accumulate both products in one accumulator; the h-side products are
+//      issued before epilogue 1 finishes, so they overlap it) -> gate math, new hidden state (epilogue 2)
+//   -> fc2 -> Q row, masked greedy choice, Philox epsilon draw, record completion (epilogue 3)
+//   -> one bulk store of the finished record per environment, episode bookkeeping, hidden-state reset.
+//
+// Thread roles: 256 epilogue threads - thread (row, half) owns one accumulator row (one agent) and 32 of its
+// 64 hidden columns, so gate math, arg-max and the random draw need no cross-thread reduction - plus one
+// control warp whose lane 0 issues every tcgen05.mma and whose lanes share the bulk copies.  The two halves
+// split the third epilogue: half 0 chooses actions while half 1 converts the next step's observations.
+// All hand-offs go through mbarriers with bounded waits; an expired wait sets MARL_STATUS_TIMEOUT and lets
+// the block run to its end without touching anything out of range.
+//
+// Shared memory: the packed weights (bf16 matrices in operand layout, fp32 bias/one-hot tables), one x/y
+// operand buffer, one hidden-state operand buffer, two sets of ring records (double-buffered over steps).
+#include <cstring>
+#include <vector>
+
 #include "common.cuh"
+#include "tcgen05.cuh"
 
 namespace marl {
-bool tc_supported(int, int, int, int, int) { return false; }
-size_t tc_wpack_bytes(int, int, int, int) { return 0; }
-void tc_pack_weights(int, int, int, int, const float*, const float*, const float*, const float*, const float*,
-                     const float*, const float*, const float*, void*) {}
-void tc_tiling(int, int, int, int* ept, int* num_tiles) { *ept = 1; *num_tiles = 0; }
-int launch_actor_tc(const ActorParams&, int, cudaStream_t) { return -(int)cudaErrorNotSupported; }
+
+constexpr int TC_ROWS = 128;
+constexpr int TC_H = 64;
+constexpr int TC_EPI_THREADS = 256;
+constexpr int TC_THREADS = 288;
+constexpr int TC_TAB = 68;                 // row stride (floats) of the bias/one-hot tables
+constexpr uint32_t TC_LBO_A = 2048;        // k-chunk stride of a 128-row operand
+constexpr uint32_t TC_LBO_X = 2048 + 16;   // padded for the observation operand: spreads the converter's stores
+constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
+// tensor-memory columns
+constexpr uint32_t TM_FC1 = 0, TM_R = 64, TM_Z = 128, TM_IN = 192, TM_HN = 256, TM_Q = 320, TM_COLS = 512;
+
+struct TcLayout {
+  int32_t Dk, NQ, nchunk, ept;
+  // packed weight image (same offsets in global and shared memory)
+  uint32_t off_W1, off_Wih, off_Whh, off_W2, off_tab_id, off_tab_la, off_gb, off_b2, wbytes;
+  // shared memory only
+  uint32_t off_xy, off_hb, off_rec, off_dst, off_reset, off_la, off_bar, total;
+};
+
+static uint32_t up16(uint32_t v) { return (v + 15u) & ~15u; }
+
+static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
+  TcLayout L;
+  memset(&L, 0, sizeof(L));
+  L.Dk = (D + 15) & ~15;
+  L.NQ = A <= 16 ? 16 : 32;
+  L.nchunk = L.Dk / 8;
+  L.ept = TC_ROWS / n;
+  uint32_t o = 0;
+  L.off_W1 = o; o += (uint32_t)L.nchunk * TC_H * 16;
+  L.off_Wih = o; o += 8u * 3 * TC_H * 16;
+  L.off_Whh = o; o += 8u * 3 * TC_H * 16;
+  L.off_W2 = o; o += 8u * L.NQ * 16;
+  L.off_tab_id = o; o += up16(sizeof(float) * n * TC_TAB);
+  L.off_tab_la = o; o += up16(sizeof(float) * A * TC_TAB);
+  L.off_gb = o; o += sizeof(float) * 4 * TC_H;
+  L.off_b2 = o; o += sizeof(float) * 32;
+  L.wbytes = o;
+  const uint32_t xbytes = (uint32_t)L.nchunk * TC_LBO_X;
+  L.off_xy = o; o += up16(xbytes > 8 * TC_LBO_A ? xbytes : 8 * TC_LBO_A);
+  L.off_hb = o; o += 8 * TC_LBO_A;
+  L.off_rec = o; o += 2u * L.ept * (uint32_t)rec_bytes;
+  L.off_dst = o; o += 2u * TC_ROWS * 8;
+  L.off_reset = o; o += TC_ROWS * 4;
+  L.off_la = o; o += TC_ROWS * 4;
+  L.off_bar = o; o += 128;
+  L.total = o;
+  return L;
+}
+
+static int rec_bytes_of(int n, int D, int A) {
+  auto up = [](size_t v) { return (v + 15) / 16 * 16; };
+  return (int)(up(4 * (size_t)n * D) + up((size_t)n * A) + up(4 * (size_t)n) + up(4 * (size_t)n * A) + 16);
+}
+
+bool tc_supported(int n, int D, int A, int H, int prec) {
+  if (prec != MARL_PRECISION_BF16 || H != TC_H) return false;
+  if (D % 8 != 0 || D > 256 || n < 1 || n > 32 || A < 1 || A > 32) return false;
+  return tc_layout(n, D, A, rec_bytes_of(n, D, A)).total <= TC_SMEM_MAX;
+}
+
+size_t tc_wpack_bytes(int n, int D, int A, int H) {
+  if (H != TC_H || D % 8 != 0) return 0;
+  return tc_layout(n, D, A, rec_bytes_of(n, D, A)).wbytes;
+}
+
+static uint16_t bf16_bits(float v) {
+  uint32_t u;
+  memcpy(&u, &v, 4);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x40);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+static float bf16_value(float v) {
+  const uint32_t u = (uint32_t)bf16_bits(v) << 16;
+  float o;
+  memcpy(&o, &u, 4);
+  return o;
+}
+
+// Element (row, k) of an N-row K-major operand: k-chunks of all rows are contiguous (LBO = N * 16).
+static size_t operand_offset(int N, int row, int k) { return (size_t)(k / 8) * N * 16 + (size_t)row * 16 + (k % 8) * 2; }
+
+void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b1, const float* Wih,
+                     const float* bih, const float* Whh, const float* bhh, const float* W2, const float* b2,
+                     void* dst_host) {
+  const TcLayout L = tc_layout(n, D, A, rec_bytes_of(n, D, A));
+  const int I = D + n + A;
+  uint8_t* o = static_cast<uint8_t*>(dst_host);
+  memset(o, 0, L.wbytes);
+  auto put = [&](uint32_t base, int N, int row, int k, float v) {
+    const uint16_t b = bf16_bits(v);
+    memcpy(o + base + operand_offset(N, row, k), &b, 2);
+  };
+  for (int j = 0; j < H; ++j)
+    for (int k = 0; k < D; ++k) put(L.off_W1, H, j, k, W1[(size_t)j * I + k]);
+  for (int r = 0; r < 3 * H; ++r)
+    for (int k = 0; k < H; ++k) {
+      put(L.off_Wih, 3 * H, r, k, Wih[(size_t)r * H + k]);
+      put(L.off_Whh, 3 * H, r, k, Whh[(size_t)r * H + k]);
+    }
+  for (int a = 0; a < A; ++a)
+    for (int k = 0; k < H; ++k) put(L.off_W2, L.NQ, a, k, W2[(size_t)a * H + k]);
+  float* tid_ = reinterpret_cast<float*>(o + L.off_tab_id);
+  float* tla = reinterpret_cast<float*>(o + L.off_tab_la);
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < H; ++j) tid_[i * TC_TAB + j] = b1[j] + bf16_value(W1[(size_t)j * I + D + i]);
+  for (int a = 0; a < A; ++a)
+    for (int j = 0; j < H; ++j) tla[a * TC_TAB + j] = bf16_value(W1[(size_t)j * I + D + n + a]);
+  float* gb = reinterpret_cast<float*>(o + L.off_gb);
+  for (int j = 0; j < H; ++j) {
+    gb[j] = bih[j] + bhh[j];
+    gb[H + j] = bih[H + j] + bhh[H + j];
+    gb[2 * H + j] = bih[2 * H + j];
+    gb[3 * H + j] = bhh[2 * H + j];
+  }
+  float* pb2 = reinterpret_cast<float*>(o + L.off_b2);
+  for (int a = 0; a < A; ++a) pb2[a] = b2[a];
+}
+
+void tc_tiling(int E, int n, int /*sms*/, int* ept, int* num_tiles) {
+  *ept = TC_ROWS / n;
+  *num_tiles = (E + *ept - 1) / *ept;
+}
+
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float sigmoid_fast(float x) { return fmaf(0.5f, tanh_fast(0.5f * x), 0.5f); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+struct TcBars {
+  uint64_t full[2], xready, fc1d, yready, grud, hready, fc2d, stepd, wload;
+  uint32_t tmem_base, abort;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+    actor_tc_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TcLayout L) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  using namespace tc;
+  TcBars* B = reinterpret_cast<TcBars*>(smem + L.off_bar);
+  uint8_t* xy = smem + L.off_xy;
+  uint8_t* hb = smem + L.off_hb;
+  uint8_t* recs = smem + L.off_rec;
+  unsigned long long* dst_s = reinterpret_cast<unsigned long long*>(smem + L.off_dst);  // [2][128]
+  int32_t* reset_s = reinterpret_cast<int32_t*>(smem + L.off_reset);
+  int32_t* la_s = reinterpret_cast<int32_t*>(smem + L.off_la);
+  const float* tab_id = reinterpret_cast<const float*>(smem + L.off_tab_id);
+  const float* tab_la = reinterpret_cast<const float*>(smem + L.off_tab_la);
+  const float* gb = reinterpret_cast<const float*>(smem + L.off_gb);
+  const float* b2s = reinterpret_cast<const float*>(smem + L.off_b2);
+  volatile uint32_t* abortf = &B->abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n = p.n, D = p.D, A = p.A;
+  const uint32_t rec_bytes = p.rl.rec_bytes;
+  const uint32_t buf_bytes = (uint32_t)L.ept * rec_bytes;
+
+  if (tid == 0) {
+    mbar_init(&B->full[0], 1);
+    mbar_init(&B->full[1], 1);
+    mbar_init(&B->xready, 128);
+    mbar_init(&B->fc1d, 1);
+    mbar_init(&B->yready, 256);
+    mbar_init(&B->grud, 1);
+    mbar_init(&B->hready, 256);
+    mbar_init(&B->fc2d, 1);
+    mbar_init(&B->stepd, 256);
+    mbar_init(&B->wload, 1);
+    B->abort = 0;
+    mbar_init_fence();
+  }
+  if (warp == 8) tmem_alloc(&B->tmem_base, TM_COLS);
+  // record buffers start as zeros so that the padding bytes of every stored record are zero
+  for (uint32_t i = tid; i < 2u * buf_bytes / 16u; i += TC_THREADS) reinterpret_cast<uint4*>(recs)[i] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = B->tmem_base;
+  if (tid == TC_EPI_THREADS) {
+    mbar_arrive_expect_tx(&B->wload, L.wbytes);
+    bulk_load(smem, p.wpack, L.wbytes, &B->wload);
+  }
+  mbar_wait(&B->wload, 0, abortf);
+
+  uint32_t it = 0;  // steps processed so far by this block (all tiles): parity source of the per-step barriers
+  uint32_t sd = 0;  // phases of the step_done barrier
+
+  if (warp == 8) {
+    // =========================== control warp ===========================
+    const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, L.NQ);
+    const uint32_t a_xy = smem_u32(xy), a_hb = smem_u32(hb);
+    const uint32_t a_W1 = smem_u32(smem + L.off_W1), a_Wih = smem_u32(smem + L.off_Wih);
+    const uint32_t a_Whh = smem_u32(smem + L.off_Whh), a_W2 = smem_u32(smem + L.off_W2);
+    const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)L.NQ * 16;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const int e0 = tile * L.ept;
+      const int ne = min(L.ept, p.E - e0);
+      auto issue_loads = [&](int s, uint32_t b) {
+        // the records last stored from this buffer must have left shared memory
+        bulk_wait_read_all();
+        __syncwarp();
+        const uint32_t env_bytes = (uint32_t)(n * D) * 4u;
+        if (lane == 0) mbar_arrive_expect_tx(&B->full[b], env_bytes * (uint32_t)ne);
+        __syncwarp();
+        const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
+        for (int el = lane; el < ne; el += 32)
+          bulk_load(recs + b * buf_bytes + (uint32_t)el * rec_bytes, src + (size_t)el * n * D, env_bytes, &B->full[b]);
+      };
+      issue_loads(0, it & 1);
+      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden operand in place
+      ++sd;
+      for (int s = 0; s < p.T; ++s) {
+        const uint32_t b = it & 1, par = it & 1;
+        mbar_wait(&B->xready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+          for (int ks = 0; ks < L.Dk / 16; ++ks)
+            mma_bf16(tmem + TM_FC1, smem_desc(a_xy + ks * 2 * TC_LBO_X, TC_LBO_X, 128),
+                     smem_desc(a_W1 + ks * 2 * lbo_w1, lbo_w1, 128), id64, ks > 0);
+          mma_commit(&B->fc1d);
+          // h-side gate products: do not depend on this step's fc1, overlap epilogue 1
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t ad = smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
+            mma_bf16(tmem + TM_R, ad, smem_desc(a_Whh + ks * 2 * lbo_g, lbo_g, 128), id128, ks > 0);
+            mma_bf16(tmem + TM_HN, ad, smem_desc(a_Whh + 2 * TC_H * 16 + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
+          }
+        }
+        __syncwarp();
+        if (s + 1 < p.T) issue_loads(s + 1, b ^ 1);
+        mbar_wait(&B->yready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t ad = smem_desc(a_xy + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
+            mma_bf16(tmem + TM_R, ad, smem_desc(a_Wih + ks * 2 * lbo_g, lbo_g, 128), id128, 1);
+            mma_bf16(tmem + TM_IN, ad, smem_desc(a_Wih + 2 * TC_H * 16 + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
+          }
+          mma_commit(&B->grud);
+        }
+        __syncwarp();
+        mbar_wait(&B->hready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+          for (int ks = 0; ks < 4; ++ks)
+            mma_bf16(tmem + TM_Q, smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128),
+                     smem_desc(a_W2 + ks * 2 * lbo_q, lbo_q, 128), idq, ks > 0);
+          mma_commit(&B->fc2d);
+        }
+        __syncwarp();
+        mbar_wait(&B->stepd, sd & 1, abortf);  // records complete, hidden operand reset where needed
+        ++sd;
+        tc_fence_after_sync();
+        for (int el = lane; el < ne; el += 32) {
+          const unsigned long long dst = dst_s[b * TC_ROWS + el];
+          if (dst) bulk_store(reinterpret_cast<void*>(dst), recs + b * buf_bytes + (uint32_t)el * rec_bytes, rec_bytes);
+        }
+        bulk_commit();
+        ++it;
+      }
+    }
+    bulk_wait_all();
+  } else {
+    // =========================== epilogue threads ===========================
+    const int row = tid & 127, half = tid >> 7;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const int el = row / n, ai = row - el * n;
+    const int cb = half * 32;  // first hidden column of this thread
+    unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
+    uint32_t st_bits = 0;
+    float h[32];
+
+    // converts the observations of the record buffer `b` into the bf16 operand (threads of half 1)
+    auto convert_x = [&](uint32_t b, int R) {
+      const int items = TC_ROWS * L.nchunk;
+      for (int j = row; j < items; j += 128) {
+        const int r = j / L.nchunk, c = j - r * L.nchunk;
+        uint4 o = make_uint4(0, 0, 0, 0);
+        if (r < R && c * 8 < D) {
+          const int rel = r / n, ra = r - rel * n;
+          const float4* src =
+              reinterpret_cast<const float4*>(recs + b * buf_bytes + (uint32_t)rel * rec_bytes + (uint32_t)(ra * D + c * 8) * 4u);
+          const float4 v0 = src[0], v1 = src[1];
+          o.x = pack_bf16x2(v0.x, v0.y);
+          o.y = pack_bf16x2(v0.z, v0.w);
+          o.z = pack_bf16x2(v1.x, v1.y);
+          o.w = pack_bf16x2(v1.z, v1.w);
+        }
+        *reinterpret_cast<uint4*>(xy + (uint32_t)c * TC_LBO_X + (uint32_t)r * 16u) = o;
+      }
+    };
+
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const int e0 = tile * L.ept;
+      const int ne = min(L.ept, p.E - e0);
+      const int R = ne * n;
+      const bool live = row < R;
+      const bool is_row = live && half == 0;             // owner of the row's choice
+      const bool is_env = is_row && ai == 0;             // owner of the environment's cursor
+      const int e = e0 + el;
+      const size_t grow = (size_t)e * n + ai;             // global row
+      int32_t slot = 0, pos = 0, ok = 0;
+      long long epc = 0;
+
+      // ---- tile prologue ----
+      {
+        const float4* src = reinterpret_cast<const float4*>(p.h + grow * TC_H + cb);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float4 v = live ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          h[4 * q] = v.x; h[4 * q + 1] = v.y; h[4 * q + 2] = v.z; h[4 * q + 3] = v.w;
+        }
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 o = make_uint4(pack_bf16x2(h[8 * cc], h[8 * cc + 1]), pack_bf16x2(h[8 * cc + 2], h[8 * cc + 3]),
+                                     pack_bf16x2(h[8 * cc + 4], h[8 * cc + 5]), pack_bf16x2(h[8 * cc + 6], h[8 * cc + 7]));
+          *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+        }
+        if (half == 0) la_s[row] = live ? p.last_action[grow] : -1;
+        if (half == 0) reset_s[row] = 0;
+        if (is_env) {
+          slot = p.slot[e];
+          pos = p.pos[e];
+          epc = p.ep_count[e];
+          ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
+          if (!ok) st_bits |= MARL_STATUS_BAD_INDEX;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&B->stepd);
+        if (half == 1) {
+          mbar_wait(&B->full[it & 1], (it >> 1) & 1, abortf);
+          convert_x(it & 1, R);
+          fence_proxy_async_smem();
+          mbar_arrive(&B->xready);
+        }
+      }
+
+      for (int s = 0; s < p.T; ++s) {
+        const uint32_t b = it & 1, par = it & 1;
+        const uint32_t t = p.t0 + (uint32_t)s;
+        const float eps = eps_at(p, t);
+        uint8_t* rec = recs + b * buf_bytes + (uint32_t)el * rec_bytes;  // this row's environment record
+
+        // ---- early global loads of the step (latency hidden behind epilogues 1 and 2) ----
+        uint32_t mask = 0;
+        float reward = 0.f;
+        int done = 0;
+        if (is_row) {
+          const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + grow * A;
+          for (int a = 0; a < A; ++a) mask |= (av[a] ? 1u : 0u) << a;
+        }
+        if (is_env) {
+          reward = p.reward[(size_t)s * p.env_step_stride + e];
+          done = p.done[(size_t)s * p.env_step_stride + e] ? 1 : 0;
+          unsigned long long dst = 0;
+          if (ok) {
+            dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
+            if (pos == 0) {  // an episode opens in this slot
+              p.slot_epid[slot] = epc * (long long)p.E + e;
+              p.slot_len[slot] = 0;
+              p.slot_complete[slot] = 0;
+            }
+          }
+          dst_s[b * TC_ROWS + el] = dst;
+        }
+
+        // ---- epilogue 1: y = relu(fc1 + b1 + W1[:, id] + W1[:, last]) -> bf16 operand ----
+        mbar_wait(&B->fc1d, par, abortf);
+        tc_fence_after_sync();
+        {
+          const int last = la_s[row];
+          const float* tid_row = tab_id + ai * TC_TAB + cb;
+          const float* tla_row = tab_la + (last >= 0 ? last : 0) * TC_TAB + cb;
+#pragma unroll
+          for (int c16 = 0; c16 < 2; ++c16) {
+            uint32_t v[16];
+            tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
+            tmem_ld_wait();
+            float y[16];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float4 a4 = *reinterpret_cast<const float4*>(tid_row + c16 * 16 + 4 * q);
+              float4 l4 = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (last >= 0) l4 = *reinterpret_cast<const float4*>(tla_row + c16 * 16 + 4 * q);
+              y[4 * q] = fmaxf(__uint_as_float(v[4 * q]) + a4.x + l4.x, 0.f);
+              y[4 * q + 1] = fmaxf(__uint_as_float(v[4 * q + 1]) + a4.y + l4.y, 0.f);
+              y[4 * q + 2] = fmaxf(__uint_as_float(v[4 * q + 2]) + a4.z + l4.z, 0.f);
+              y[4 * q + 3] = fmaxf(__uint_as_float(v[4 * q + 3]) + a4.w + l4.w, 0.f);
+            }
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+              const uint4 o = make_uint4(pack_bf16x2(y[8 * cc], y[8 * cc + 1]), pack_bf16x2(y[8 * cc + 2], y[8 * cc + 3]),
+                                         pack_bf16x2(y[8 * cc + 4], y[8 * cc + 5]), pack_bf16x2(y[8 * cc + 6], y[8 * cc + 7]));
+              *reinterpret_cast<uint4*>(xy + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+            }
+          }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&B->yready);
+
+        // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand ----
+        mbar_wait(&B->grud, par, abortf);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int c16 = 0; c16 < 2; ++c16) {
+          uint32_t vr[16], vz[16], vi[16], vh[16];
+          const uint32_t col = (uint32_t)(cb + c16 * 16);
+          tmem_ld16(tmem + lane_addr + TM_R + col, vr);
+          tmem_ld16(tmem + lane_addr + TM_Z + col, vz);
+          tmem_ld16(tmem + lane_addr + TM_IN + col, vi);
+          tmem_ld16(tmem + lane_addr + TM_HN + col, vh);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 br = *reinterpret_cast<const float4*>(gb + col + 4 * q);
+            const float4 bz = *reinterpret_cast<const float4*>(gb + TC_H + col + 4 * q);
+            const float4 bi = *reinterpret_cast<const float4*>(gb + 2 * TC_H + col + 4 * q);
+            const float4 bh = *reinterpret_cast<const float4*>(gb + 3 * TC_H + col + 4 * q);
+            const float brv[4] = {br.x, br.y, br.z, br.w}, bzv[4] = {bz.x, bz.y, bz.z, bz.w};
+            const float biv[4] = {bi.x, bi.y, bi.z, bi.w}, bhv[4] = {bh.x, bh.y, bh.z, bh.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int j = 4 * q + u;
+              const float rg = sigmoid_fast(__uint_as_float(vr[j]) + brv[u]);
+              const float zg = sigmoid_fast(__uint_as_float(vz[j]) + bzv[u]);
+              const float cand = tanh_fast(fmaf(rg, __uint_as_float(vh[j]) + bhv[u], __uint_as_float(vi[j]) + biv[u]));
+              const float hp = h[c16 * 16 + j];
+              h[c16 * 16 + j] = fmaf(zg, hp - cand, cand);  // (1 - z) * cand + z * h
+            }
+          }
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const float* hv = h + c16 * 16 + 8 * cc;
+            const uint4 o = make_uint4(pack_bf16x2(hv[0], hv[1]), pack_bf16x2(hv[2], hv[3]), pack_bf16x2(hv[4], hv[5]),
+                                       pack_bf16x2(hv[6], hv[7]));
+            *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+          }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&B->hready);
+
+        // ---- epilogue 3: half 0 chooses and records; half 1 prepares the next step's operand ----
+        if (half == 0) {
+          mbar_wait(&B->fc2d, par, abortf);
+          tc_fence_after_sync();
+          uint32_t vq[32];
+          {
+            uint32_t(&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(vq);
+            tmem_ld16(tmem + lane_addr + TM_Q, lo);
+            if (L.NQ == 32) {
+              uint32_t(&hi)[16] = *reinterpret_cast<uint32_t(*)[16]>(vq + 16);
+              tmem_ld16(tmem + lane_addr + TM_Q + 16, hi);
+            }
+            tmem_ld_wait();
+          }
+          tc_fence_before_sync();
+          if (is_row) {
+            float* qrow = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
+#pragma unroll
+            for (int a = 0; a < 32; ++a)
+              if (a < A && a < L.NQ) qrow[a] = __uint_as_float(vq[a]) + b2s[a];
+            uint32_t flags;
+            const int act = select_action([&](int a) { return qrow[a]; }, A, mask, eps, p.seed, t, (uint32_t)e,
+                                          (uint32_t)ai, flags);
+            c_steps += 1;
+            c_explore += flags & 1u;
+            if (flags & 2u) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
+            la_s[row] = act;
+            reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
+            uint8_t* avd = rec + p.rl.off_avail + ai * A;
+            for (int a = 0; a < A; ++a) avd[a] = (uint8_t)((mask >> a) & 1u);
+            const int tk = p.trace_first + s;
+            if (tk < p.trace_cap) {
+              const size_t trow = ((size_t)tk * p.E + e) * n + ai;
+              if (p.trace_actions) p.trace_actions[trow] = act;
+              if (p.trace_q)
+                for (int a = 0; a < A; ++a) p.trace_q[trow * A + a] = qrow[a];
+            }
+            if (p.actions_out && s == p.T - 1) p.actions_out[grow] = act;
+          }
+          if (is_env) {
+            int closed = 0;
+            if (ok) {
+              *reinterpret_cast<float*>(rec + p.rl.off_reward) = reward;
+              rec[p.rl.off_done] = (uint8_t)done;
+              if (done || pos + 1 == p.L) {
+                p.slot_len[slot] = pos + 1;
+                p.slot_complete[slot] = 1;
+                c_episodes += 1;
+                if (!done) c_trunc += 1;
+                epc += 1;
+                slot = e * p.S + (int)(epc % p.S);
+                pos = 0;
+                closed = 1;
+              } else {
+                pos += 1;
+              }
+            }
+            reset_s[el] = closed;
+          }
+        } else if (s + 1 < p.T) {
+          mbar_wait(&B->full[b ^ 1], ((it + 1) >> 1) & 1, abortf);
+          convert_x(b ^ 1, R);
+          fence_proxy_async_smem();
+          mbar_arrive(&B->xready);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // ---- a closed episode restarts from a zero hidden state and no last action ----
+        if (live && reset_s[el]) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) h[j] = 0.f;
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc)
+            *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = make_uint4(0, 0, 0, 0);
+          if (half == 0) la_s[row] = -1;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&B->stepd);
+        ++it;
+      }
+
+      // ---- tile epilogue: state back to global memory ----
+      if (live) {
+        float4* dsth = reinterpret_cast<float4*>(p.h + grow * TC_H + cb);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) dsth[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
+      }
+      if (is_row) p.last_action[grow] = la_s[row];
+      if (is_env && ok) {
+        p.slot[e] = slot;
+        p.pos[e] = pos;
+        p.ep_count[e] = epc;
+        if (pos > 0) p.slot_len[slot] = pos;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s / reset_s are rewritten by the next tile's prologue
+    }
+    if (c_steps) atomicAdd(p.counters + CNT_AGENT_STEPS, c_steps);
+    if (c_explore) atomicAdd(p.counters + CNT_EXPLORED, c_explore);
+    if (c_noavail) atomicAdd(p.counters + CNT_NO_AVAIL, c_noavail);
+    if (c_episodes) atomicAdd(p.counters + CNT_EPISODES, c_episodes);
+    if (c_trunc) atomicAdd(p.counters + CNT_TRUNCATED, c_trunc);
+    if (st_bits) atomicOr(p.status, st_bits);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && B->abort) atomicOr(p.status, MARL_STATUS_TIMEOUT);
+  if (warp == 8) tmem_dealloc(tmem, TM_COLS);
+}
+
+// Returns the number of kernels launched or a negative cudaError.
+int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream) {
+  const TcLayout L = tc_layout(p.n, p.D, p.A, (int)p.rl.rec_bytes);
+  if (reinterpret_cast<uintptr_t>(p.obs) % 16) return -(int)cudaErrorMisalignedAddress;
+  static uint32_t configured = 0;
+  if (L.total > configured) {
+    const cudaError_t e = cudaFuncSetAttribute(actor_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+    if (e != cudaSuccess) return -(int)e;
+    configured = L.total;
+  }
+  int grid = p.num_tiles < sms ? p.num_tiles : sms;
+  if (grid < 1) grid = 1;
+  actor_tc_kernel<<<grid, TC_THREADS, L.total, stream>>>(p, L);
+  const cudaError_t err = cudaGetLastError();
+  return err == cudaSuccess ? 1 : -(int)err;
+}
+
 }  // namespace marl

@@ -270,9 +270,9 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
     delete a;
     return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
   }
-  // Small batches leave most SMs without a 128-row tile: the FFMA kernel spreads them better.
+  // Below a couple of 128-row tiles the FFMA kernel, which spreads 64-row tiles over more SMs, is used.
   a->use_tc = cfg->kernel == MARL_KERNEL_TENSOR ||
-              (cfg->kernel == MARL_KERNEL_AUTO && tc_ok && (long long)cfg->n_envs * cfg->n_agents >= 128LL * a->sms);
+              (cfg->kernel == MARL_KERNEL_AUTO && tc_ok && (long long)cfg->n_envs * cfg->n_agents >= 256);
 
   auto bind = [&](void* mem, size_t have, size_t need, uint8_t** dst, bool* own, const char* what) -> int {
     if (mem) {

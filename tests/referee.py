@@ -21,6 +21,10 @@ import oracle
 from paper_2205_05248_b200 import binding, workloads
 
 RTOL = {"fp32": 1e-5, "bf16": 2e-2}
+# Share of greedy decisions that may be near-ties.  fp32 path: the two sides differ by accumulation order
+# (about 1e-6 in Q).  bf16 path: operand roundings can flip and the kernel uses the hardware tanh
+# approximation, so Q differs by about 1e-3 and proportionally more decisions fall inside the tie band.
+NEAR_TIE_BUDGET = {"fp32": 1e-4, "bf16": 2e-3}
 
 
 def row_rel_err(got: np.ndarray, want: np.ndarray) -> np.ndarray:
@@ -48,12 +52,14 @@ def run_gpu_rollout(cfg, weights, kernel="auto", T=None, splits=None, want_q=Tru
     return actor, acts, q
 
 
-def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=1e-4, n_threads=None):
+def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=None, n_threads=None):
     """Checks parts 1-4 for the listed environments (default: all).  Returns a summary dict."""
     T = cfg["T"] if T is None else T
     E, n, A, H = cfg["E"], cfg["n"], cfg["A"], cfg["H"]
     ids = np.arange(E) if env_ids is None else np.asarray(env_ids)
     rtol = RTOL[cfg["precision"]]
+    if near_tie_budget is None:
+        near_tie_budget = NEAR_TIE_BUDGET[cfg["precision"]]
     tids = torch.as_tensor(ids, device=gpu_actions.device, dtype=torch.long)
     g_act = gpu_actions[:T].index_select(1, tids).cpu().numpy()
     g_q = gpu_q[:T].index_select(1, tids).cpu().numpy()

@@ -69,8 +69,8 @@ def test_configs_2_to_4_parity(k, n_ids):
     actor.destroy()
 
 
-@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "ffma"), (128, "bf16", "ffma"), (64, "fp32", "ffma"),
-                                           (128, "fp32", "ffma")])
+@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "tensor"), (64, "bf16", "ffma"), (128, "bf16", "ffma"),
+                                           (64, "fp32", "ffma"), (128, "fp32", "ffma")])
 def test_config5_parity_small_E(H, prec, kernel):
     cfg = workloads.config(5, E=4096, H=H, precision=prec)
     cfg["T"] = 24
@@ -92,11 +92,24 @@ def test_ragged_tiles_and_tiny_shapes():
         actor.destroy()
 
 
-def test_done_every_step_and_never():
-    for thr, L in ((1 << 24, 4), (0, 5)):
-        cfg = workloads.small_config(H=64, E=40, C=80, L=L, T=17, env=dict(done_thresh24=thr))
+def test_tensor_kernel_ragged_tiles_and_tiny_shapes():
+    """The tcgen05 kernel on tile tails, agent counts that do not divide 128, one row, 32 actions."""
+    for over in (dict(E=37, n=5, D=16, C=74), dict(E=1, n=1, A=1, D=8, C=2), dict(E=150, n=7, A=32, D=24, C=150),
+                 dict(E=9, n=32, A=2, D=40, C=9), dict(E=300, n=3, D=96, C=300), dict(E=130, n=8, D=80, A=14, C=260)):
+        cfg = workloads.small_config(H=64, L=7, T=20, precision="bf16", **over)
         w = workloads.make_weights(cfg)
-        actor, acts, q = run_gpu_rollout(cfg, w, kernel="ffma")
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="tensor")
+        res = referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
+        assert res["kernel"] == "tcgen05"
+        actor.destroy()
+
+
+@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
+def test_done_every_step_and_never(kernel, prec):
+    for thr, L in ((1 << 24, 4), (0, 5)):
+        cfg = workloads.small_config(H=64, D=8, E=40, C=80, L=L, T=17, precision=prec, env=dict(done_thresh24=thr))
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
         res = referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
         _, counters = actor.status()
         if thr:
@@ -106,23 +119,25 @@ def test_done_every_step_and_never():
         actor.destroy()
 
 
-def test_annealed_epsilon_and_split_rollouts_resume():
+@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
+def test_annealed_epsilon_and_split_rollouts_resume(kernel, prec):
     """eps schedule follows the global step; rollout(T) == rollout(a) + rollout(b); a checkpoint restored
     into a fresh handle continues identically."""
-    cfg = workloads.small_config(H=64, E=64, C=128, L=9, T=30, eps_start=1.0, eps_end=0.05, anneal_steps=29)
+    cfg = workloads.small_config(H=64, D=16, E=64, C=128, L=9, T=30, eps_start=1.0, eps_end=0.05, anneal_steps=29,
+                                 precision=prec)
     w = workloads.make_weights(cfg)
-    one, a1, q1 = run_gpu_rollout(cfg, w, kernel="ffma")
+    one, a1, q1 = run_gpu_rollout(cfg, w, kernel=kernel)
     referee(cfg, w, one, a1, q1, near_tie_budget=2e-3)
-    two, a2, q2 = run_gpu_rollout(cfg, w, kernel="ffma", splits=[11, 19])
+    two, a2, q2 = run_gpu_rollout(cfg, w, kernel=kernel, splits=[11, 19])
     assert torch.equal(a1, a2) and torch.equal(q1, q2)
     r1, r2 = one.ring_view(), two.ring_view()
     assert torch.equal(one.ring_mem, two.ring_mem)
     # checkpoint after 11 steps -> fresh handle -> 19 more
-    first = binding.Actor(cfg, kernel="ffma")
+    first = binding.Actor(cfg, kernel=kernel)
     first.set_weights(w)
     first.rollout(cfg["env"], 11, 1.0, 0.05, 29)
     st = first.get_state()
-    second = binding.Actor(cfg, kernel="ffma")
+    second = binding.Actor(cfg, kernel=kernel)
     second.set_weights(w)
     second.ring_mem.copy_(first.ring_mem)
     second.set_state(st)
@@ -137,16 +152,17 @@ def test_annealed_epsilon_and_split_rollouts_resume():
         a.destroy()
 
 
-def test_step_api_equals_rollout_and_host_variant():
+@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
+def test_step_api_equals_rollout_and_host_variant(kernel, prec):
     """T calls of marl_actor_step (device inputs) and of marl_actor_step_host (host inputs) reproduce
     marl_rollout: same actions, same ring, same state."""
-    cfg = workloads.small_config(H=64, E=50, n=4, C=100, L=8, T=12)
+    cfg = workloads.small_config(H=64, D=24, E=50, n=4, C=100, L=8, T=12, precision=prec)
     w = workloads.make_weights(cfg)
-    ref, acts, q = run_gpu_rollout(cfg, w, kernel="ffma")
+    ref, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
     obs, avail, rew, done = ref.env_generate(cfg["env"], 0, cfg["T"])
-    dev = binding.Actor(cfg, kernel="ffma")
+    dev = binding.Actor(cfg, kernel=kernel)
     dev.set_weights(w)
-    host = binding.Actor(cfg, kernel="ffma")
+    host = binding.Actor(cfg, kernel=kernel)
     host.set_weights(w)
     h_obs, h_avail, h_rew, h_done = [t.cpu().pin_memory() for t in (obs, avail, rew, done)]
     h_act = torch.empty((cfg["E"], cfg["n"]), dtype=torch.int32).pin_memory()
