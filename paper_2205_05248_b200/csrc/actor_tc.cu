@@ -36,7 +36,6 @@ constexpr int TC_ROWS = 128;
 constexpr int TC_H = 64;
 constexpr int TC_EPI_THREADS = 256;
 constexpr int TC_THREADS = 288;
-constexpr int TC_TAB = 68;                 // row stride (floats) of the bias/one-hot tables
 constexpr uint32_t TC_LBO_A = 2048;        // k-chunk stride of a 128-row operand
 constexpr uint32_t TC_LBO_X = 2048 + 16;   // padded for the observation operand: spreads the converter's stores
 constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
@@ -44,13 +43,22 @@ constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
 constexpr uint32_t TM_FC1 = 0, TM_R = 64, TM_Z = 128, TM_IN = 192, TM_HN = 256, TM_Q = 320, TM_COLS = 512;
 
 struct TcLayout {
-  int32_t Dk, NQ, nchunk, ept;
+  int32_t Dk, NQ, nchunk, ept, ohK, ohc;
   // packed weight image (same offsets in global and shared memory)
-  uint32_t off_W1, off_Wih, off_Whh, off_W2, off_tab_id, off_tab_la, off_gb, off_b2, wbytes;
+  uint32_t off_W1, off_Wih, off_Bin, off_Whh, off_W2, wbytes;
   // shared memory only
-  uint32_t off_xy, off_hb, off_rec, off_dst, off_reset, off_la, off_bar, total;
+  uint32_t off_xy, off_hb, off_oh, off_rec, off_dst, off_reset, off_rowoff, off_bar, total;
 };
 
+// Operand K-columns beyond the data columns ("extension"): the fp32 biases and the two one-hot parts of
+// the network input enter the GEMMs as extra K columns, so the epilogues add nothing.
+//   one-hot operand tile (A side, per row):  col 0..2 = 1, col 3+i = [agent == i], col 3+n+a = [last action == a]
+//   fc1 weights (B side):    k = Dk+0..2: b1 split into three bf16 pieces (their sum is b1 to fp32 accuracy),
+//                            k = Dk+3+i: W1[:, D+i],  k = Dk+3+n+a: W1[:, D+n+a]
+//   W_hh, W2, and a small tile for the candidate gate's input bias: bias pieces at k = 64..66 (resp. 0..2),
+//   multiplied by the three ones of the one-hot tile; all other extension entries are zero.
+// The reset and update rows of W_ih / W_hh and their biases are stored halved (exact in bf16), so that
+// sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 needs no multiply in the epilogue.
 static uint32_t up16(uint32_t v) { return (v + 15u) & ~15u; }
 
 static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
@@ -60,23 +68,23 @@ static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
   L.NQ = A <= 16 ? 16 : 32;
   L.nchunk = L.Dk / 8;
   L.ept = TC_ROWS / n;
+  L.ohK = (3 + n + A + 15) & ~15;
+  L.ohc = L.ohK / 8;
   uint32_t o = 0;
-  L.off_W1 = o; o += (uint32_t)L.nchunk * TC_H * 16;
+  L.off_W1 = o; o += (uint32_t)(L.nchunk + L.ohc) * TC_H * 16;
   L.off_Wih = o; o += 8u * 3 * TC_H * 16;
-  L.off_Whh = o; o += 8u * 3 * TC_H * 16;
-  L.off_W2 = o; o += 8u * L.NQ * 16;
-  L.off_tab_id = o; o += up16(sizeof(float) * n * TC_TAB);
-  L.off_tab_la = o; o += up16(sizeof(float) * A * TC_TAB);
-  L.off_gb = o; o += sizeof(float) * 4 * TC_H;
-  L.off_b2 = o; o += sizeof(float) * 32;
+  L.off_Bin = o; o += 2u * TC_H * 16;
+  L.off_Whh = o; o += 10u * 3 * TC_H * 16;
+  L.off_W2 = o; o += 10u * L.NQ * 16;
   L.wbytes = o;
   const uint32_t xbytes = (uint32_t)L.nchunk * TC_LBO_X;
   L.off_xy = o; o += up16(xbytes > 8 * TC_LBO_A ? xbytes : 8 * TC_LBO_A);
   L.off_hb = o; o += 8 * TC_LBO_A;
+  L.off_oh = o; o += (uint32_t)L.ohc * TC_LBO_A;
   L.off_rec = o; o += 2u * L.ept * (uint32_t)rec_bytes;
   L.off_dst = o; o += 2u * TC_ROWS * 8;
   L.off_reset = o; o += TC_ROWS * 4;
-  L.off_la = o; o += TC_ROWS * 4;
+  L.off_rowoff = o; o += TC_ROWS * 4;
   L.off_bar = o; o += 128;
   L.total = o;
   return L;
@@ -94,7 +102,7 @@ bool tc_supported(int n, int D, int A, int H, int prec) {
 }
 
 size_t tc_wpack_bytes(int n, int D, int A, int H) {
-  if (H != TC_H || D % 8 != 0) return 0;
+  if (H != TC_H || D % 8 != 0 || n < 1 || n > 32 || A < 1 || A > 32) return 0;
   return tc_layout(n, D, A, rec_bytes_of(n, D, A)).wbytes;
 }
 
@@ -126,30 +134,35 @@ void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b
     const uint16_t b = bf16_bits(v);
     memcpy(o + base + operand_offset(N, row, k), &b, 2);
   };
-  for (int j = 0; j < H; ++j)
-    for (int k = 0; k < D; ++k) put(L.off_W1, H, j, k, W1[(size_t)j * I + k]);
-  for (int r = 0; r < 3 * H; ++r)
-    for (int k = 0; k < H; ++k) {
-      put(L.off_Wih, 3 * H, r, k, Wih[(size_t)r * H + k]);
-      put(L.off_Whh, 3 * H, r, k, Whh[(size_t)r * H + k]);
-    }
-  for (int a = 0; a < A; ++a)
-    for (int k = 0; k < H; ++k) put(L.off_W2, L.NQ, a, k, W2[(size_t)a * H + k]);
-  float* tid_ = reinterpret_cast<float*>(o + L.off_tab_id);
-  float* tla = reinterpret_cast<float*>(o + L.off_tab_la);
-  for (int i = 0; i < n; ++i)
-    for (int j = 0; j < H; ++j) tid_[i * TC_TAB + j] = b1[j] + bf16_value(W1[(size_t)j * I + D + i]);
-  for (int a = 0; a < A; ++a)
-    for (int j = 0; j < H; ++j) tla[a * TC_TAB + j] = bf16_value(W1[(size_t)j * I + D + n + a]);
-  float* gb = reinterpret_cast<float*>(o + L.off_gb);
+  // a fp32 value as three bf16 pieces at k0, k0+1, k0+2
+  auto put3 = [&](uint32_t base, int N, int row, int k0, float v) {
+    const float p0 = bf16_value(v), p1 = bf16_value(v - p0), p2 = bf16_value(v - p0 - p1);
+    put(base, N, row, k0, p0);
+    put(base, N, row, k0 + 1, p1);
+    put(base, N, row, k0 + 2, p2);
+  };
   for (int j = 0; j < H; ++j) {
-    gb[j] = bih[j] + bhh[j];
-    gb[H + j] = bih[H + j] + bhh[H + j];
-    gb[2 * H + j] = bih[2 * H + j];
-    gb[3 * H + j] = bhh[2 * H + j];
+    for (int k = 0; k < D; ++k) put(L.off_W1, H, j, k, W1[(size_t)j * I + k]);
+    put3(L.off_W1, H, j, L.Dk, b1[j]);
+    for (int i = 0; i < n + A; ++i) put(L.off_W1, H, j, L.Dk + 3 + i, W1[(size_t)j * I + D + i]);
   }
-  float* pb2 = reinterpret_cast<float*>(o + L.off_b2);
-  for (int a = 0; a < A; ++a) pb2[a] = b2[a];
+  for (int r = 0; r < 3 * H; ++r) {
+    const float sc = r < 2 * H ? 0.5f : 1.0f;  // reset and update rows are stored halved
+    for (int k = 0; k < H; ++k) {
+      put(L.off_Wih, 3 * H, r, k, sc * bf16_value(Wih[(size_t)r * H + k]));
+      put(L.off_Whh, 3 * H, r, k, sc * bf16_value(Whh[(size_t)r * H + k]));
+    }
+    if (r < 2 * H) {
+      put3(L.off_Whh, 3 * H, r, H, 0.5f * (bih[r] + bhh[r]));
+    } else {
+      put3(L.off_Whh, 3 * H, r, H, bhh[r]);
+      put3(L.off_Bin, H, r - 2 * H, 0, bih[r]);
+    }
+  }
+  for (int a = 0; a < A; ++a) {
+    for (int k = 0; k < H; ++k) put(L.off_W2, L.NQ, a, k, W2[(size_t)a * H + k]);
+    put3(L.off_W2, L.NQ, a, H, b2[a]);
+  }
 }
 
 void tc_tiling(int E, int n, int /*sms*/, int* ept, int* num_tiles) {
@@ -181,14 +194,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   TcBars* B = reinterpret_cast<TcBars*>(smem + L.off_bar);
   uint8_t* xy = smem + L.off_xy;
   uint8_t* hb = smem + L.off_hb;
+  uint8_t* oh = smem + L.off_oh;
   uint8_t* recs = smem + L.off_rec;
   unsigned long long* dst_s = reinterpret_cast<unsigned long long*>(smem + L.off_dst);  // [2][128]
   int32_t* reset_s = reinterpret_cast<int32_t*>(smem + L.off_reset);
-  int32_t* la_s = reinterpret_cast<int32_t*>(smem + L.off_la);
-  const float* tab_id = reinterpret_cast<const float*>(smem + L.off_tab_id);
-  const float* tab_la = reinterpret_cast<const float*>(smem + L.off_tab_la);
-  const float* gb = reinterpret_cast<const float*>(smem + L.off_gb);
-  const float* b2s = reinterpret_cast<const float*>(smem + L.off_b2);
+  uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(smem + L.off_rowoff);
   volatile uint32_t* abortf = &B->abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -213,6 +223,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   if (warp == 8) tmem_alloc(&B->tmem_base, TM_COLS);
   // record buffers start as zeros so that the padding bytes of every stored record are zero
   for (uint32_t i = tid; i < 2u * buf_bytes / 16u; i += TC_THREADS) reinterpret_cast<uint4*>(recs)[i] = make_uint4(0, 0, 0, 0);
+  if (tid < TC_ROWS) rowoff_s[tid] = (uint32_t)(tid / n) * rec_bytes + (uint32_t)((tid % n) * D) * 4u;
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -230,10 +241,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   if (warp == 8) {
     // =========================== control warp ===========================
     const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, L.NQ);
-    const uint32_t a_xy = smem_u32(xy), a_hb = smem_u32(hb);
+    const uint32_t a_xy = smem_u32(xy), a_hb = smem_u32(hb), a_oh = smem_u32(oh);
     const uint32_t a_W1 = smem_u32(smem + L.off_W1), a_Wih = smem_u32(smem + L.off_Wih);
     const uint32_t a_Whh = smem_u32(smem + L.off_Whh), a_W2 = smem_u32(smem + L.off_W2);
+    const uint32_t a_Bin = smem_u32(smem + L.off_Bin);
     const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)L.NQ * 16;
+    const uint32_t gate_n = 2 * TC_H * 16;  // byte offset of the candidate-gate rows inside a k-chunk of W_ih / W_hh
+    const uint64_t d_ones = smem_desc(a_oh, TC_LBO_A, 128);  // the 16 columns that hold the three ones
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
       const int ne = min(L.ept, p.E - e0);
@@ -249,23 +263,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           bulk_load(recs + b * buf_bytes + (uint32_t)el * rec_bytes, src + (size_t)el * n * D, env_bytes, &B->full[b]);
       };
       issue_loads(0, it & 1);
-      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden operand in place
+      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden and one-hot operands in place
       ++sd;
       for (int s = 0; s < p.T; ++s) {
         const uint32_t b = it & 1, par = it & 1;
         mbar_wait(&B->xready, par, abortf);
         tc_fence_after_sync();
         if (lane == 0) {
+          // fc1: observation columns, then the one-hot / bias columns
           for (int ks = 0; ks < L.Dk / 16; ++ks)
             mma_bf16(tmem + TM_FC1, smem_desc(a_xy + ks * 2 * TC_LBO_X, TC_LBO_X, 128),
                      smem_desc(a_W1 + ks * 2 * lbo_w1, lbo_w1, 128), id64, ks > 0);
+          for (int ks = 0; ks < L.ohK / 16; ++ks)
+            mma_bf16(tmem + TM_FC1, smem_desc(a_oh + ks * 2 * TC_LBO_A, TC_LBO_A, 128),
+                     smem_desc(a_W1 + (L.nchunk + ks * 2) * lbo_w1, lbo_w1, 128), id64, 1);
           mma_commit(&B->fc1d);
-          // h-side gate products: do not depend on this step's fc1, overlap epilogue 1
+          // h-side gate products and all gate biases: independent of this step's fc1, overlap epilogue 1
           for (int ks = 0; ks < 4; ++ks) {
             const uint64_t ad = smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
             mma_bf16(tmem + TM_R, ad, smem_desc(a_Whh + ks * 2 * lbo_g, lbo_g, 128), id128, ks > 0);
-            mma_bf16(tmem + TM_HN, ad, smem_desc(a_Whh + 2 * TC_H * 16 + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
+            mma_bf16(tmem + TM_HN, ad, smem_desc(a_Whh + gate_n + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
           }
+          mma_bf16(tmem + TM_R, d_ones, smem_desc(a_Whh + 8 * lbo_g, lbo_g, 128), id128, 1);
+          mma_bf16(tmem + TM_HN, d_ones, smem_desc(a_Whh + gate_n + 8 * lbo_g, lbo_g, 128), id64, 1);
         }
         __syncwarp();
         if (s + 1 < p.T) issue_loads(s + 1, b ^ 1);
@@ -275,8 +295,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           for (int ks = 0; ks < 4; ++ks) {
             const uint64_t ad = smem_desc(a_xy + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
             mma_bf16(tmem + TM_R, ad, smem_desc(a_Wih + ks * 2 * lbo_g, lbo_g, 128), id128, 1);
-            mma_bf16(tmem + TM_IN, ad, smem_desc(a_Wih + 2 * TC_H * 16 + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
+            mma_bf16(tmem + TM_IN, ad, smem_desc(a_Wih + gate_n + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
           }
+          mma_bf16(tmem + TM_IN, d_ones, smem_desc(a_Bin, lbo_w1, 128), id64, 1);
           mma_commit(&B->grud);
         }
         __syncwarp();
@@ -286,10 +307,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           for (int ks = 0; ks < 4; ++ks)
             mma_bf16(tmem + TM_Q, smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128),
                      smem_desc(a_W2 + ks * 2 * lbo_q, lbo_q, 128), idq, ks > 0);
+          mma_bf16(tmem + TM_Q, d_ones, smem_desc(a_W2 + 8 * lbo_q, lbo_q, 128), idq, 1);
           mma_commit(&B->fc2d);
         }
         __syncwarp();
-        mbar_wait(&B->stepd, sd & 1, abortf);  // records complete, hidden operand reset where needed
+        mbar_wait(&B->stepd, sd & 1, abortf);  // records complete, operands updated for the next step
         ++sd;
         tc_fence_after_sync();
         for (int el = lane; el < ne; el += 32) {
@@ -307,6 +329,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const int el = row / n, ai = row - el * n;
     const int cb = half * 32;  // first hidden column of this thread
+    const uint32_t inv_nchunk = 0xFFFFFFFFu / (uint32_t)L.nchunk + 1u;  // j / nchunk == umulhi(j, inv) for j < 2^16
     unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
     uint32_t st_bits = 0;
     float h[32];
@@ -314,13 +337,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     // converts the observations of the record buffer `b` into the bf16 operand (threads of half 1)
     auto convert_x = [&](uint32_t b, int R) {
       const int items = TC_ROWS * L.nchunk;
+      const uint8_t* base = recs + b * buf_bytes;
       for (int j = row; j < items; j += 128) {
-        const int r = j / L.nchunk, c = j - r * L.nchunk;
+        const int r = (int)__umulhi((uint32_t)j, inv_nchunk), c = j - r * L.nchunk;
         uint4 o = make_uint4(0, 0, 0, 0);
         if (r < R && c * 8 < D) {
-          const int rel = r / n, ra = r - rel * n;
-          const float4* src =
-              reinterpret_cast<const float4*>(recs + b * buf_bytes + (uint32_t)rel * rec_bytes + (uint32_t)(ra * D + c * 8) * 4u);
+          const float4* src = reinterpret_cast<const float4*>(base + rowoff_s[r] + (uint32_t)c * 32u);
           const float4 v0 = src[0], v1 = src[1];
           o.x = pack_bf16x2(v0.x, v0.y);
           o.y = pack_bf16x2(v0.z, v0.w);
@@ -330,6 +352,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         *reinterpret_cast<uint4*>(xy + (uint32_t)c * TC_LBO_X + (uint32_t)r * 16u) = o;
       }
     };
+    // one-hot operand tile of this thread's row: byte address of column k
+    auto oh_col = [&](int k) { return oh + (uint32_t)(k >> 3) * TC_LBO_A + (uint32_t)row * 16u + (uint32_t)(k & 7) * 2u; };
 
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
@@ -340,8 +364,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const bool is_env = is_row && ai == 0;             // owner of the environment's cursor
       const int e = e0 + el;
       const size_t grow = (size_t)e * n + ai;             // global row
-      int32_t slot = 0, pos = 0, ok = 0;
+      int32_t slot = 0, pos = 0, ok = 0, la = -1;
       long long epc = 0;
+      uint32_t av_raw[32];      // availability bytes of the coming step (row owners)
+      float reward_raw = 0.f;   // reward / done of the coming step (environment owners)
+      uint32_t done_raw = 0;
 
       // ---- tile prologue ----
       {
@@ -357,14 +384,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                                      pack_bf16x2(h[8 * cc + 4], h[8 * cc + 5]), pack_bf16x2(h[8 * cc + 6], h[8 * cc + 7]));
           *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
         }
-        if (half == 0) la_s[row] = live ? p.last_action[grow] : -1;
-        if (half == 0) reset_s[row] = 0;
+        if (half == 0) {
+          reset_s[row] = 0;
+          for (int c = 0; c < L.ohc; ++c)
+            *reinterpret_cast<uint4*>(oh + (uint32_t)c * TC_LBO_A + (uint32_t)row * 16u) = make_uint4(0, 0, 0, 0);
+        }
+        if (is_row) {
+          la = p.last_action[grow];
+          *reinterpret_cast<uint16_t*>(oh_col(0)) = 0x3F80;  // bf16 1.0: the three bias columns
+          *reinterpret_cast<uint16_t*>(oh_col(1)) = 0x3F80;
+          *reinterpret_cast<uint16_t*>(oh_col(2)) = 0x3F80;
+          *reinterpret_cast<uint16_t*>(oh_col(3 + ai)) = 0x3F80;
+          if (la >= 0 && la < A) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0x3F80;
+          const uint8_t* av = p.avail + grow * A;
+#pragma unroll
+          for (int a = 0; a < 32; ++a)
+            if (a < A) av_raw[a] = av[a];
+        }
         if (is_env) {
           slot = p.slot[e];
           pos = p.pos[e];
           epc = p.ep_count[e];
           ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
           if (!ok) st_bits |= MARL_STATUS_BAD_INDEX;
+          reward_raw = p.reward[e];
+          done_raw = p.done[e];
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -383,17 +427,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const float eps = eps_at(p, t);
         uint8_t* rec = recs + b * buf_bytes + (uint32_t)el * rec_bytes;  // this row's environment record
 
-        // ---- early global loads of the step (latency hidden behind epilogues 1 and 2) ----
+        // ---- this step's availability bytes were requested one step ahead; request the next step's now, so
+        //      that no global-load latency sits on the step's critical path ----
         uint32_t mask = 0;
-        float reward = 0.f;
-        int done = 0;
         if (is_row) {
-          const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + grow * A;
-          for (int a = 0; a < A; ++a) mask |= (av[a] ? 1u : 0u) << a;
+#pragma unroll
+          for (int a = 0; a < 32; ++a)
+            if (a < A) mask |= (av_raw[a] ? 1u : 0u) << a;
+          if (s + 1 < p.T) {
+            const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
+#pragma unroll
+            for (int a = 0; a < 32; ++a)
+              if (a < A) av_raw[a] = av[a];
+          }
         }
+        const float reward = reward_raw;
+        const int done = done_raw ? 1 : 0;
         if (is_env) {
-          reward = p.reward[(size_t)s * p.env_step_stride + e];
-          done = p.done[(size_t)s * p.env_step_stride + e] ? 1 : 0;
+          if (s + 1 < p.T) {
+            reward_raw = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
+            done_raw = p.done[(size_t)(s + 1) * p.env_step_stride + e];
+          }
           unsigned long long dst = 0;
           if (ok) {
             dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
@@ -406,42 +460,30 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           dst_s[b * TC_ROWS + el] = dst;
         }
 
-        // ---- epilogue 1: y = relu(fc1 + b1 + W1[:, id] + W1[:, last]) -> bf16 operand ----
+        // ---- epilogue 1: y = relu(fc1) -> bf16 operand (bias and one-hot columns are inside the GEMM) ----
         mbar_wait(&B->fc1d, par, abortf);
         tc_fence_after_sync();
-        {
-          const int last = la_s[row];
-          const float* tid_row = tab_id + ai * TC_TAB + cb;
-          const float* tla_row = tab_la + (last >= 0 ? last : 0) * TC_TAB + cb;
 #pragma unroll
-          for (int c16 = 0; c16 < 2; ++c16) {
-            uint32_t v[16];
-            tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
-            tmem_ld_wait();
-            float y[16];
+        for (int c16 = 0; c16 < 2; ++c16) {
+          uint32_t v[16];
+          tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
+          tmem_ld_wait();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 a4 = *reinterpret_cast<const float4*>(tid_row + c16 * 16 + 4 * q);
-              float4 l4 = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (last >= 0) l4 = *reinterpret_cast<const float4*>(tla_row + c16 * 16 + 4 * q);
-              y[4 * q] = fmaxf(__uint_as_float(v[4 * q]) + a4.x + l4.x, 0.f);
-              y[4 * q + 1] = fmaxf(__uint_as_float(v[4 * q + 1]) + a4.y + l4.y, 0.f);
-              y[4 * q + 2] = fmaxf(__uint_as_float(v[4 * q + 2]) + a4.z + l4.z, 0.f);
-              y[4 * q + 3] = fmaxf(__uint_as_float(v[4 * q + 3]) + a4.w + l4.w, 0.f);
-            }
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-              const uint4 o = make_uint4(pack_bf16x2(y[8 * cc], y[8 * cc + 1]), pack_bf16x2(y[8 * cc + 2], y[8 * cc + 3]),
-                                         pack_bf16x2(y[8 * cc + 4], y[8 * cc + 5]), pack_bf16x2(y[8 * cc + 6], y[8 * cc + 7]));
-              *reinterpret_cast<uint4*>(xy + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
-            }
+          for (int cc = 0; cc < 2; ++cc) {
+            const uint32_t* w = v + 8 * cc;
+            const uint4 o = make_uint4(pack_bf16x2(fmaxf(__uint_as_float(w[0]), 0.f), fmaxf(__uint_as_float(w[1]), 0.f)),
+                                       pack_bf16x2(fmaxf(__uint_as_float(w[2]), 0.f), fmaxf(__uint_as_float(w[3]), 0.f)),
+                                       pack_bf16x2(fmaxf(__uint_as_float(w[4]), 0.f), fmaxf(__uint_as_float(w[5]), 0.f)),
+                                       pack_bf16x2(fmaxf(__uint_as_float(w[6]), 0.f), fmaxf(__uint_as_float(w[7]), 0.f)));
+            *reinterpret_cast<uint4*>(xy + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
           }
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&B->yready);
 
-        // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand ----
+        // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand.
+        //      The r and z accumulators hold half the pre-activation: sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 ----
         mbar_wait(&B->grud, par, abortf);
         tc_fence_after_sync();
 #pragma unroll
@@ -454,22 +496,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           tmem_ld16(tmem + lane_addr + TM_HN + col, vh);
           tmem_ld_wait();
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float4 br = *reinterpret_cast<const float4*>(gb + col + 4 * q);
-            const float4 bz = *reinterpret_cast<const float4*>(gb + TC_H + col + 4 * q);
-            const float4 bi = *reinterpret_cast<const float4*>(gb + 2 * TC_H + col + 4 * q);
-            const float4 bh = *reinterpret_cast<const float4*>(gb + 3 * TC_H + col + 4 * q);
-            const float brv[4] = {br.x, br.y, br.z, br.w}, bzv[4] = {bz.x, bz.y, bz.z, bz.w};
-            const float biv[4] = {bi.x, bi.y, bi.z, bi.w}, bhv[4] = {bh.x, bh.y, bh.z, bh.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int j = 4 * q + u;
-              const float rg = sigmoid_fast(__uint_as_float(vr[j]) + brv[u]);
-              const float zg = sigmoid_fast(__uint_as_float(vz[j]) + bzv[u]);
-              const float cand = tanh_fast(fmaf(rg, __uint_as_float(vh[j]) + bhv[u], __uint_as_float(vi[j]) + biv[u]));
-              const float hp = h[c16 * 16 + j];
-              h[c16 * 16 + j] = fmaf(zg, hp - cand, cand);  // (1 - z) * cand + z * h
-            }
+          for (int j = 0; j < 16; ++j) {
+            const float rg = fmaf(0.5f, tanh_fast(__uint_as_float(vr[j])), 0.5f);
+            const float zg = fmaf(0.5f, tanh_fast(__uint_as_float(vz[j])), 0.5f);
+            const float cand = tanh_fast(fmaf(rg, __uint_as_float(vh[j]), __uint_as_float(vi[j])));
+            const float hp = h[c16 * 16 + j];
+            h[c16 * 16 + j] = fmaf(zg, hp - cand, cand);  // (1 - z) * cand + z * h
           }
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
@@ -487,29 +519,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         if (half == 0) {
           mbar_wait(&B->fc2d, par, abortf);
           tc_fence_after_sync();
-          uint32_t vq[32];
-          {
-            uint32_t(&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(vq);
-            tmem_ld16(tmem + lane_addr + TM_Q, lo);
-            if (L.NQ == 32) {
-              uint32_t(&hi)[16] = *reinterpret_cast<uint32_t(*)[16]>(vq + 16);
-              tmem_ld16(tmem + lane_addr + TM_Q + 16, hi);
-            }
-            tmem_ld_wait();
+          uint32_t qlo[16], qhi[16];
+          tmem_ld16(tmem + lane_addr + TM_Q, qlo);
+          if (L.NQ == 32) {
+            tmem_ld16(tmem + lane_addr + TM_Q + 16, qhi);
+          } else {
+#pragma unroll
+            for (int a = 0; a < 16; ++a) qhi[a] = 0;
           }
+          tmem_ld_wait();
           tc_fence_before_sync();
           if (is_row) {
             float* qrow = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
 #pragma unroll
-            for (int a = 0; a < 32; ++a)
-              if (a < A && a < L.NQ) qrow[a] = __uint_as_float(vq[a]) + b2s[a];
+            for (int a = 0; a < 16; ++a)
+              if (a < A) qrow[a] = __uint_as_float(qlo[a]);
+#pragma unroll
+            for (int a = 0; a < 16; ++a)
+              if (16 + a < A) qrow[16 + a] = __uint_as_float(qhi[a]);
             uint32_t flags;
             const int act = select_action([&](int a) { return qrow[a]; }, A, mask, eps, p.seed, t, (uint32_t)e,
                                           (uint32_t)ai, flags);
             c_steps += 1;
             c_explore += flags & 1u;
             if (flags & 2u) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
-            la_s[row] = act;
+            if (act != la) {  // move the last-action one-hot
+              if (la >= 0) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
+              *reinterpret_cast<uint16_t*>(oh_col(3 + n + act)) = 0x3F80;
+              la = act;
+            }
             reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
             uint8_t* avd = rec + p.rl.off_avail + ai * A;
             for (int a = 0; a < A; ++a) avd[a] = (uint8_t)((mask >> a) & 1u);
@@ -556,7 +594,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
           for (int cc = 0; cc < 4; ++cc)
             *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = make_uint4(0, 0, 0, 0);
-          if (half == 0) la_s[row] = -1;
+          if (half == 0 && la >= 0) {
+            *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
+            la = -1;
+          }
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -570,14 +611,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
         for (int q = 0; q < 8; ++q) dsth[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
       }
-      if (is_row) p.last_action[grow] = la_s[row];
+      if (is_row) p.last_action[grow] = la;
       if (is_env && ok) {
         p.slot[e] = slot;
         p.pos[e] = pos;
         p.ep_count[e] = epc;
         if (pos > 0) p.slot_len[slot] = pos;
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s / reset_s are rewritten by the next tile's prologue
+      asm volatile("bar.sync 1, 256;" ::: "memory");  // reset_s is rewritten by the next tile's prologue
     }
     if (c_steps) atomicAdd(p.counters + CNT_AGENT_STEPS, c_steps);
     if (c_explore) atomicAdd(p.counters + CNT_EXPLORED, c_explore);
