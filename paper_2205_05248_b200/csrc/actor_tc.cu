@@ -17,7 +17,7 @@
 //
 // Thread roles: 256 epilogue threads - thread (row, half) owns one accumulator row (one agent) and 32 of its
 // 64 hidden columns, so gate math, arg-max and the random draw need no cross-thread reduction - plus one
-// control warp whose lane 0 issues every tcgen05.mma and whose lanes share the bulk copies.  The two halves
+// warp whose lane 0 issues every tcgen05.mma and one warp whose lanes share the bulk copies.  The two halves
 // split the third epilogue: half 0 chooses actions while half 1 converts the next step's observations.
 // All hand-offs go through mbarriers with bounded waits; an expired wait sets MARL_STATUS_TIMEOUT and lets
 // the block run to its end without touching anything out of range.
@@ -35,7 +35,11 @@ namespace marl {
 constexpr int TC_ROWS = 128;
 constexpr int TC_H = 64;
 constexpr int TC_EPI_THREADS = 256;
-constexpr int TC_THREADS = 288;
+constexpr int TC_THREADS = 384;  // two epilogue warpgroups + one service warpgroup (MMA warp, copy warp, two idle)
+// Register split after start-up (setmaxnreg): the block is launched with 168 registers per thread
+// (384 * 168 = 64512); the service warpgroup drops to 88 and each epilogue warpgroup rises to 208:
+// 256 * 208 + 128 * 88 = 64512, exactly the launch total.
+constexpr int TC_REGS_EPILOGUE = 208, TC_REGS_SERVICE = 88;
 constexpr uint32_t TC_LBO_A = 2048;        // k-chunk stride of a 128-row operand
 constexpr uint32_t TC_LBO_X = 2048 + 16;   // padded for the observation operand: spreads the converter's stores
 constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
@@ -238,22 +242,84 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   uint32_t it = 0;  // steps processed so far by this block (all tiles): parity source of the per-step barriers
   uint32_t sd = 0;  // phases of the step_done barrier
 
-  if (warp == 8) {
-    // =========================== control warp ===========================
+  if (warp >= 8) {
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(TC_REGS_SERVICE));
+   if (warp == 8) {
+    // =========================== MMA warp: lane 0 issues every tcgen05.mma ===========================
     const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, L.NQ);
-    const uint32_t a_xy = smem_u32(xy), a_hb = smem_u32(hb), a_oh = smem_u32(oh);
-    const uint32_t a_W1 = smem_u32(smem + L.off_W1), a_Wih = smem_u32(smem + L.off_Wih);
-    const uint32_t a_Whh = smem_u32(smem + L.off_Whh), a_W2 = smem_u32(smem + L.off_W2);
-    const uint32_t a_Bin = smem_u32(smem + L.off_Bin);
     const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)L.NQ * 16;
     const uint32_t gate_n = 2 * TC_H * 16;  // byte offset of the candidate-gate rows inside a k-chunk of W_ih / W_hh
-    const uint64_t d_ones = smem_desc(a_oh, TC_LBO_A, 128);  // the 16 columns that hold the three ones
+    // descriptors of the first k-step of every operand; a later k-step adds (2 * LBO) >> 4 to the address field
+    const uint64_t d_x = smem_desc(smem_u32(xy), TC_LBO_X, 128), d_y = smem_desc(smem_u32(xy), TC_LBO_A, 128);
+    const uint64_t d_h = smem_desc(smem_u32(hb), TC_LBO_A, 128), d_oh = smem_desc(smem_u32(oh), TC_LBO_A, 128);
+    const uint64_t d_W1 = smem_desc(smem_u32(smem + L.off_W1), lbo_w1, 128);
+    const uint64_t d_W1oh = smem_desc(smem_u32(smem + L.off_W1) + (uint32_t)L.nchunk * lbo_w1, lbo_w1, 128);
+    const uint64_t d_Wih = smem_desc(smem_u32(smem + L.off_Wih), lbo_g, 128);
+    const uint64_t d_Wih_n = smem_desc(smem_u32(smem + L.off_Wih) + gate_n, lbo_g, 128);
+    const uint64_t d_Whh = smem_desc(smem_u32(smem + L.off_Whh), lbo_g, 128);
+    const uint64_t d_Whh_n = smem_desc(smem_u32(smem + L.off_Whh) + gate_n, lbo_g, 128);
+    const uint64_t d_Bin = smem_desc(smem_u32(smem + L.off_Bin), lbo_w1, 128);
+    const uint64_t d_W2 = smem_desc(smem_u32(smem + L.off_W2), lbo_q, 128);
+    const uint64_t k_x = (2 * TC_LBO_X) >> 4, k_a = (2 * TC_LBO_A) >> 4, k_w1 = (2 * lbo_w1) >> 4, k_g = (2 * lbo_g) >> 4,
+                   k_q = (2 * lbo_q) >> 4;
+    const int ks_obs = L.Dk / 16, ks_oh = L.ohK / 16;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden and one-hot operands in place
+      ++sd;
+      for (int s = 0; s < p.T; ++s) {
+        const uint32_t par = it & 1;
+        mbar_wait(&B->xready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+          // fc1: observation columns, then the one-hot / bias columns
+          for (int ks = 0; ks < ks_obs; ++ks) mma_bf16(tmem + TM_FC1, d_x + ks * k_x, d_W1 + ks * k_w1, id64, ks > 0);
+          for (int ks = 0; ks < ks_oh; ++ks) mma_bf16(tmem + TM_FC1, d_oh + ks * k_a, d_W1oh + ks * k_w1, id64, 1);
+          mma_commit(&B->fc1d);
+          // h-side gate products and all gate biases: independent of this step's fc1, overlap epilogue 1
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            mma_bf16(tmem + TM_R, d_h + ks * k_a, d_Whh + ks * k_g, id128, ks > 0);
+            mma_bf16(tmem + TM_HN, d_h + ks * k_a, d_Whh_n + ks * k_g, id64, ks > 0);
+          }
+          mma_bf16(tmem + TM_R, d_oh, d_Whh + 4 * k_g, id128, 1);
+          mma_bf16(tmem + TM_HN, d_oh, d_Whh_n + 4 * k_g, id64, 1);
+        }
+        __syncwarp();
+        mbar_wait(&B->yready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            mma_bf16(tmem + TM_R, d_y + ks * k_a, d_Wih + ks * k_g, id128, 1);
+            mma_bf16(tmem + TM_IN, d_y + ks * k_a, d_Wih_n + ks * k_g, id64, ks > 0);
+          }
+          mma_bf16(tmem + TM_IN, d_oh, d_Bin, id64, 1);
+          mma_commit(&B->grud);
+        }
+        __syncwarp();
+        mbar_wait(&B->hready, par, abortf);
+        tc_fence_after_sync();
+        if (lane == 0) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) mma_bf16(tmem + TM_Q, d_h + ks * k_a, d_W2 + ks * k_q, idq, ks > 0);
+          mma_bf16(tmem + TM_Q, d_oh, d_W2 + 4 * k_q, idq, 1);
+          mma_commit(&B->fc2d);
+        }
+        __syncwarp();
+        mbar_wait(&B->stepd, sd & 1, abortf);  // operands updated for the next step
+        ++sd;
+        ++it;
+      }
+    }
+  } else if (warp == 9) {
+    // =========================== copy warp: bulk loads of observations, bulk stores of records ==============
+    // Observations of step i (counted over all tiles of this block) land in record buffer i & 1; they are
+    // requested two steps ahead, as soon as the records of step i - 2 have been stored from that buffer.
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
       const int ne = min(L.ept, p.E - e0);
       auto issue_loads = [&](int s, uint32_t b) {
-        // the records last stored from this buffer must have left shared memory
-        bulk_wait_read_all();
+        bulk_wait_read_all();  // this lane's earlier stores have left shared memory
         __syncwarp();
         const uint32_t env_bytes = (uint32_t)(n * D) * 4u;
         if (lane == 0) mbar_arrive_expect_tx(&B->full[b], env_bytes * (uint32_t)ne);
@@ -263,67 +329,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           bulk_load(recs + b * buf_bytes + (uint32_t)el * rec_bytes, src + (size_t)el * n * D, env_bytes, &B->full[b]);
       };
       issue_loads(0, it & 1);
-      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden and one-hot operands in place
+      if (p.T > 1) issue_loads(1, (it + 1) & 1);
+      mbar_wait(&B->stepd, sd & 1, abortf);  // the tile prologue's phase
       ++sd;
       for (int s = 0; s < p.T; ++s) {
-        const uint32_t b = it & 1, par = it & 1;
-        mbar_wait(&B->xready, par, abortf);
-        tc_fence_after_sync();
-        if (lane == 0) {
-          // fc1: observation columns, then the one-hot / bias columns
-          for (int ks = 0; ks < L.Dk / 16; ++ks)
-            mma_bf16(tmem + TM_FC1, smem_desc(a_xy + ks * 2 * TC_LBO_X, TC_LBO_X, 128),
-                     smem_desc(a_W1 + ks * 2 * lbo_w1, lbo_w1, 128), id64, ks > 0);
-          for (int ks = 0; ks < L.ohK / 16; ++ks)
-            mma_bf16(tmem + TM_FC1, smem_desc(a_oh + ks * 2 * TC_LBO_A, TC_LBO_A, 128),
-                     smem_desc(a_W1 + (L.nchunk + ks * 2) * lbo_w1, lbo_w1, 128), id64, 1);
-          mma_commit(&B->fc1d);
-          // h-side gate products and all gate biases: independent of this step's fc1, overlap epilogue 1
-          for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t ad = smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
-            mma_bf16(tmem + TM_R, ad, smem_desc(a_Whh + ks * 2 * lbo_g, lbo_g, 128), id128, ks > 0);
-            mma_bf16(tmem + TM_HN, ad, smem_desc(a_Whh + gate_n + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
-          }
-          mma_bf16(tmem + TM_R, d_ones, smem_desc(a_Whh + 8 * lbo_g, lbo_g, 128), id128, 1);
-          mma_bf16(tmem + TM_HN, d_ones, smem_desc(a_Whh + gate_n + 8 * lbo_g, lbo_g, 128), id64, 1);
-        }
-        __syncwarp();
-        if (s + 1 < p.T) issue_loads(s + 1, b ^ 1);
-        mbar_wait(&B->yready, par, abortf);
-        tc_fence_after_sync();
-        if (lane == 0) {
-          for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t ad = smem_desc(a_xy + ks * 2 * TC_LBO_A, TC_LBO_A, 128);
-            mma_bf16(tmem + TM_R, ad, smem_desc(a_Wih + ks * 2 * lbo_g, lbo_g, 128), id128, 1);
-            mma_bf16(tmem + TM_IN, ad, smem_desc(a_Wih + gate_n + ks * 2 * lbo_g, lbo_g, 128), id64, ks > 0);
-          }
-          mma_bf16(tmem + TM_IN, d_ones, smem_desc(a_Bin, lbo_w1, 128), id64, 1);
-          mma_commit(&B->grud);
-        }
-        __syncwarp();
-        mbar_wait(&B->hready, par, abortf);
-        tc_fence_after_sync();
-        if (lane == 0) {
-          for (int ks = 0; ks < 4; ++ks)
-            mma_bf16(tmem + TM_Q, smem_desc(a_hb + ks * 2 * TC_LBO_A, TC_LBO_A, 128),
-                     smem_desc(a_W2 + ks * 2 * lbo_q, lbo_q, 128), idq, ks > 0);
-          mma_bf16(tmem + TM_Q, d_ones, smem_desc(a_W2 + 8 * lbo_q, lbo_q, 128), idq, 1);
-          mma_commit(&B->fc2d);
-        }
-        __syncwarp();
-        mbar_wait(&B->stepd, sd & 1, abortf);  // records complete, operands updated for the next step
+        const uint32_t b = it & 1;
+        mbar_wait(&B->stepd, sd & 1, abortf);  // records of step s complete
         ++sd;
-        tc_fence_after_sync();
         for (int el = lane; el < ne; el += 32) {
           const unsigned long long dst = dst_s[b * TC_ROWS + el];
           if (dst) bulk_store(reinterpret_cast<void*>(dst), recs + b * buf_bytes + (uint32_t)el * rec_bytes, rec_bytes);
         }
         bulk_commit();
+        if (s + 2 < p.T) issue_loads(s + 2, b);
         ++it;
       }
     }
     bulk_wait_all();
+   }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(TC_REGS_EPILOGUE));
     // =========================== epilogue threads ===========================
     const int row = tid & 127, half = tid >> 7;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -336,20 +361,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 
     // converts the observations of the record buffer `b` into the bf16 operand (threads of half 1)
     auto convert_x = [&](uint32_t b, int R) {
-      const int items = TC_ROWS * L.nchunk;
+      const int items = TC_ROWS * L.nchunk;  // a multiple of 256: two items per pass keep four loads in flight
       const uint8_t* base = recs + b * buf_bytes;
-      for (int j = row; j < items; j += 128) {
-        const int r = (int)__umulhi((uint32_t)j, inv_nchunk), c = j - r * L.nchunk;
-        uint4 o = make_uint4(0, 0, 0, 0);
-        if (r < R && c * 8 < D) {
-          const float4* src = reinterpret_cast<const float4*>(base + rowoff_s[r] + (uint32_t)c * 32u);
-          const float4 v0 = src[0], v1 = src[1];
-          o.x = pack_bf16x2(v0.x, v0.y);
-          o.y = pack_bf16x2(v0.z, v0.w);
-          o.z = pack_bf16x2(v1.x, v1.y);
-          o.w = pack_bf16x2(v1.z, v1.w);
+      for (int j = row; j < items; j += 256) {
+        float4 v[2][2];
+        int rr[2], cc[2];
+        bool on[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int jj = j + 128 * u;
+          rr[u] = (int)__umulhi((uint32_t)jj, inv_nchunk);
+          cc[u] = jj - rr[u] * L.nchunk;
+          on[u] = rr[u] < R && cc[u] * 8 < D;
+          if (on[u]) {
+            const float4* src = reinterpret_cast<const float4*>(base + rowoff_s[rr[u]] + (uint32_t)cc[u] * 32u);
+            v[u][0] = src[0];
+            v[u][1] = src[1];
+          }
         }
-        *reinterpret_cast<uint4*>(xy + (uint32_t)c * TC_LBO_X + (uint32_t)r * 16u) = o;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          uint4 o = make_uint4(0, 0, 0, 0);
+          if (on[u]) {
+            o.x = pack_bf16x2(v[u][0].x, v[u][0].y);
+            o.y = pack_bf16x2(v[u][0].z, v[u][0].w);
+            o.z = pack_bf16x2(v[u][1].x, v[u][1].y);
+            o.w = pack_bf16x2(v[u][1].z, v[u][1].w);
+          }
+          *reinterpret_cast<uint4*>(xy + (uint32_t)cc[u] * TC_LBO_X + (uint32_t)rr[u] * 16u) = o;
+        }
       }
     };
     // one-hot operand tile of this thread's row: byte address of column k
@@ -433,7 +473,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         if (is_row) {
 #pragma unroll
           for (int a = 0; a < 32; ++a)
-            if (a < A) mask |= (av_raw[a] ? 1u : 0u) << a;
+            if (a < A) {
+              asm volatile("" : "+r"(av_raw[a]));  // keeps the byte's use here, a whole step after its load
+              mask |= (av_raw[a] ? 1u : 0u) << a;
+            }
           if (s + 1 < p.T) {
             const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
 #pragma unroll
@@ -441,6 +484,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               if (a < A) av_raw[a] = av[a];
           }
         }
+        asm volatile("" : "+f"(reward_raw), "+r"(done_raw));
         const float reward = reward_raw;
         const int done = done_raw ? 1 : 0;
         if (is_env) {
@@ -517,6 +561,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 
         // ---- epilogue 3: half 0 chooses and records; half 1 prepares the next step's operand ----
         if (half == 0) {
+          // the random branch does not depend on Q: drawn while fc2 runs
+          int pick = -1;
+          if (is_row && mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)e, (uint32_t)ai);
           mbar_wait(&B->fc2d, par, abortf);
           tc_fence_after_sync();
           uint32_t qlo[16], qhi[16];
@@ -530,6 +577,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           tmem_ld_wait();
           tc_fence_before_sync();
           if (is_row) {
+            // greedy rule on registers: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr
+            float m = -INFINITY;
+#pragma unroll
+            for (int a = 0; a < 32; ++a) {
+              const float qa = __uint_as_float(a < 16 ? qlo[a & 15] : qhi[a & 15]);
+              if (a < L.NQ && ((mask >> a) & 1u) && qa > m) m = qa;
+            }
+            const float thr = __fsub_rn(m, 1e-4f);
+            int g = __ffs(mask) - 1;
+#pragma unroll
+            for (int a = 31; a >= 0; --a) {
+              const float qa = __uint_as_float(a < 16 ? qlo[a & 15] : qhi[a & 15]);
+              if (a < L.NQ && ((mask >> a) & 1u) && qa >= thr) g = a;
+            }
+            const int act = mask == 0 ? 0 : (pick >= 0 ? pick : g);
+            c_steps += 1;
+            c_explore += pick >= 0 ? 1u : 0u;
+            if (mask == 0) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
+            if (act != la) {  // move the last-action one-hot
+              if (la >= 0) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
+              *reinterpret_cast<uint16_t*>(oh_col(3 + n + act)) = 0x3F80;
+              la = act;
+            }
             float* qrow = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
 #pragma unroll
             for (int a = 0; a < 16; ++a)
@@ -537,20 +607,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
             for (int a = 0; a < 16; ++a)
               if (16 + a < A) qrow[16 + a] = __uint_as_float(qhi[a]);
-            uint32_t flags;
-            const int act = select_action([&](int a) { return qrow[a]; }, A, mask, eps, p.seed, t, (uint32_t)e,
-                                          (uint32_t)ai, flags);
-            c_steps += 1;
-            c_explore += flags & 1u;
-            if (flags & 2u) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
-            if (act != la) {  // move the last-action one-hot
-              if (la >= 0) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
-              *reinterpret_cast<uint16_t*>(oh_col(3 + n + act)) = 0x3F80;
-              la = act;
-            }
             reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
             uint8_t* avd = rec + p.rl.off_avail + ai * A;
-            for (int a = 0; a < A; ++a) avd[a] = (uint8_t)((mask >> a) & 1u);
+#pragma unroll
+            for (int a = 0; a < 32; ++a)
+              if (a < A) avd[a] = (uint8_t)((mask >> a) & 1u);
             const int tk = p.trace_first + s;
             if (tk < p.trace_cap) {
               const size_t trow = ((size_t)tk * p.E + e) * n + ai;

@@ -106,25 +106,35 @@ __device__ __forceinline__ float eps_at(const ActorParams& p, uint32_t t) {
   return (float)__dadd_rn(p.eps_start, delta);
 }
 
+// The epsilon draw of one row: Philox block (t, e, i, tag 0); word 0 -> u in [0,1), explore iff u < eps; word 1
+// -> index among the K available actions (bit a of mask set = action a available), floor(w1 * K / 2^32).
+// Returns -1 if the row does not explore, otherwise the random action.  K == 0 never explores.
+__device__ __forceinline__ int draw_explore(uint32_t mask, float eps, uint64_t seed, uint32_t t, uint32_t e,
+                                            uint32_t i) {
+  uint32_t w[4];
+  philox_block(seed, t, e, i, 0, TAG_EPS, w);
+  const float u = (float)(w[0] >> 8) * (1.0f / 16777216.0f);
+  const int K = __popc(mask);
+  if (K == 0 || !(u < eps)) return -1;
+  const uint32_t j = __umulhi(w[1], (uint32_t)K);
+  return __fns(mask, 0, (int)j + 1);  // position of the (j+1)-th set bit, ascending
+}
+
 // Masked greedy choice with the lowest-index rule, then the epsilon draw (see marl_actor.h).
 // q: A values; mask: bit a set = available.  Returns the action; sets flags bit0 = explored,
 // bit1 = no action available.
 template <typename QGet>
 __device__ __forceinline__ int select_action(QGet q, int A, uint32_t mask, float eps, uint64_t seed, uint32_t t,
                                              uint32_t e, uint32_t i, uint32_t& flags) {
-  uint32_t w[4];
-  philox_block(seed, t, e, i, 0, TAG_EPS, w);
-  const float u = (float)(w[0] >> 8) * (1.0f / 16777216.0f);
-  const int K = __popc(mask);
   flags = 0;
-  if (K == 0) {
+  if (mask == 0) {
     flags = 2;
     return 0;
   }
-  if (u < eps) {
+  const int pick = draw_explore(mask, eps, seed, t, e, i);
+  if (pick >= 0) {
     flags = 1;
-    const uint32_t j = __umulhi(w[1], (uint32_t)K);
-    return __fns(mask, 0, (int)j + 1);  // position of the (j+1)-th set bit, ascending
+    return pick;
   }
   float m = -INFINITY;
   for (int a = 0; a < A; ++a)
