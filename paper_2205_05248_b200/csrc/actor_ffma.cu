@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           for (int a = 0; a < A; ++a) {
             const uint8_t b = av[a];
             if (b) m |= 1u << a;
-            if (es.ok) dst[a] = b ? 1 : 0;
+            if (es.ok) dst[a] = b;
           }
           masks[tid] = m;
         }

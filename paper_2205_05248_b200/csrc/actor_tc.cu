@@ -47,7 +47,7 @@ constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
 constexpr uint32_t TM_FC1 = 0, TM_R = 64, TM_Z = 128, TM_IN = 192, TM_HN = 256, TM_Q = 320, TM_COLS = 512;
 
 struct TcLayout {
-  int32_t Dk, NQ, nchunk, ept, ohK, ohc;
+  int32_t Dk, NQ, nchunk, ept, ohK, ohc, avail_bulk, pad_;
   // packed weight image (same offsets in global and shared memory)
   uint32_t off_W1, off_Wih, off_Bin, off_Whh, off_W2, wbytes;
   // shared memory only
@@ -191,6 +191,7 @@ struct TcBars {
   uint32_t tmem_base, abort;
 };
 
+template <int NQ>
 __global__ void __launch_bounds__(TC_THREADS, 1)
     actor_tc_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TcLayout L) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -246,8 +247,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(TC_REGS_SERVICE));
    if (warp == 8) {
     // =========================== MMA warp: lane 0 issues every tcgen05.mma ===========================
-    const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, L.NQ);
-    const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)L.NQ * 16;
+    const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, NQ);
+    const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)NQ * 16;
     const uint32_t gate_n = 2 * TC_H * 16;  // byte offset of the candidate-gate rows inside a k-chunk of W_ih / W_hh
     // descriptors of the first k-step of every operand; a later k-step adds (2 * LBO) >> 4 to the address field
     const uint64_t d_x = smem_desc(smem_u32(xy), TC_LBO_X, 128), d_y = smem_desc(smem_u32(xy), TC_LBO_A, 128);
@@ -263,16 +264,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     const uint64_t k_x = (2 * TC_LBO_X) >> 4, k_a = (2 * TC_LBO_A) >> 4, k_w1 = (2 * lbo_w1) >> 4, k_g = (2 * lbo_g) >> 4,
                    k_q = (2 * lbo_q) >> 4;
     const int ks_obs = L.Dk / 16, ks_oh = L.ohK / 16;
+    // The observation columns of fc1 need only the converted observations, so they are issued as soon as
+    // those are ready - for step s+1 while step s is still in its third epilogue.  The one-hot / bias columns
+    // follow once the step before has published its actions.
+    auto issue_fc1_obs = [&]() {
+      mbar_wait(&B->xready, it & 1, abortf);
+      tc_fence_after_sync();
+      if (lane == 0)
+        for (int ks = 0; ks < ks_obs; ++ks) mma_bf16(tmem + TM_FC1, d_x + ks * k_x, d_W1 + ks * k_w1, id64, ks > 0);
+      __syncwarp();
+    };
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      mbar_wait(&B->stepd, sd & 1, abortf);  // tile prologue done: hidden and one-hot operands in place
-      ++sd;
+      issue_fc1_obs();
       for (int s = 0; s < p.T; ++s) {
         const uint32_t par = it & 1;
-        mbar_wait(&B->xready, par, abortf);
+        mbar_wait(&B->stepd, sd & 1, abortf);  // prologue or previous step: hidden and one-hot operands in place
+        ++sd;
         tc_fence_after_sync();
         if (lane == 0) {
-          // fc1: observation columns, then the one-hot / bias columns
-          for (int ks = 0; ks < ks_obs; ++ks) mma_bf16(tmem + TM_FC1, d_x + ks * k_x, d_W1 + ks * k_w1, id64, ks > 0);
           for (int ks = 0; ks < ks_oh; ++ks) mma_bf16(tmem + TM_FC1, d_oh + ks * k_a, d_W1oh + ks * k_w1, id64, 1);
           mma_commit(&B->fc1d);
           // h-side gate products and all gate biases: independent of this step's fc1, overlap epilogue 1
@@ -306,10 +315,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           mma_commit(&B->fc2d);
         }
         __syncwarp();
-        mbar_wait(&B->stepd, sd & 1, abortf);  // operands updated for the next step
-        ++sd;
         ++it;
+        if (s + 1 < p.T) issue_fc1_obs();
       }
+      mbar_wait(&B->stepd, sd & 1, abortf);  // last step of the tile
+      ++sd;
     }
   } else if (warp == 9) {
     // =========================== copy warp: bulk loads of observations, bulk stores of records ==============
@@ -321,12 +331,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       auto issue_loads = [&](int s, uint32_t b) {
         bulk_wait_read_all();  // this lane's earlier stores have left shared memory
         __syncwarp();
-        const uint32_t env_bytes = (uint32_t)(n * D) * 4u;
-        if (lane == 0) mbar_arrive_expect_tx(&B->full[b], env_bytes * (uint32_t)ne);
+        const uint32_t env_bytes = (uint32_t)(n * D) * 4u, av_bytes = L.avail_bulk ? (uint32_t)(n * A) : 0u;
+        if (lane == 0) mbar_arrive_expect_tx(&B->full[b], (env_bytes + av_bytes) * (uint32_t)ne);
         __syncwarp();
         const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
-        for (int el = lane; el < ne; el += 32)
-          bulk_load(recs + b * buf_bytes + (uint32_t)el * rec_bytes, src + (size_t)el * n * D, env_bytes, &B->full[b]);
+        const uint8_t* asrc = p.avail + (size_t)s * p.avail_step_stride + (size_t)e0 * n * A;
+        for (int el = lane; el < ne; el += 32) {
+          uint8_t* r = recs + b * buf_bytes + (uint32_t)el * rec_bytes;
+          bulk_load(r, src + (size_t)el * n * D, env_bytes, &B->full[b]);
+          if (av_bytes) bulk_load(r + p.rl.off_avail, asrc + (size_t)el * av_bytes, av_bytes, &B->full[b]);
+        }
       };
       issue_loads(0, it & 1);
       if (p.T > 1) issue_loads(1, (it + 1) & 1);
@@ -436,10 +450,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           *reinterpret_cast<uint16_t*>(oh_col(2)) = 0x3F80;
           *reinterpret_cast<uint16_t*>(oh_col(3 + ai)) = 0x3F80;
           if (la >= 0 && la < A) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0x3F80;
-          const uint8_t* av = p.avail + grow * A;
+          if (!L.avail_bulk) {
+            const uint8_t* av = p.avail + grow * A;
 #pragma unroll
-          for (int a = 0; a < 32; ++a)
-            if (a < A) av_raw[a] = av[a];
+            for (int a = 0; a < 32; ++a)
+              if (a < A) av_raw[a] = av[a];
+          }
         }
         if (is_env) {
           slot = p.slot[e];
@@ -464,45 +480,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       for (int s = 0; s < p.T; ++s) {
         const uint32_t b = it & 1, par = it & 1;
         const uint32_t t = p.t0 + (uint32_t)s;
-        const float eps = eps_at(p, t);
         uint8_t* rec = recs + b * buf_bytes + (uint32_t)el * rec_bytes;  // this row's environment record
-
-        // ---- this step's availability bytes were requested one step ahead; request the next step's now, so
-        //      that no global-load latency sits on the step's critical path ----
-        uint32_t mask = 0;
-        if (is_row) {
-#pragma unroll
-          for (int a = 0; a < 32; ++a)
-            if (a < A) {
-              asm volatile("" : "+r"(av_raw[a]));  // keeps the byte's use here, a whole step after its load
-              mask |= (av_raw[a] ? 1u : 0u) << a;
-            }
-          if (s + 1 < p.T) {
-            const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
-#pragma unroll
-            for (int a = 0; a < 32; ++a)
-              if (a < A) av_raw[a] = av[a];
-          }
-        }
-        asm volatile("" : "+f"(reward_raw), "+r"(done_raw));
-        const float reward = reward_raw;
-        const int done = done_raw ? 1 : 0;
-        if (is_env) {
-          if (s + 1 < p.T) {
-            reward_raw = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
-            done_raw = p.done[(size_t)(s + 1) * p.env_step_stride + e];
-          }
-          unsigned long long dst = 0;
-          if (ok) {
-            dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
-            if (pos == 0) {  // an episode opens in this slot
-              p.slot_epid[slot] = epc * (long long)p.E + e;
-              p.slot_len[slot] = 0;
-              p.slot_complete[slot] = 0;
-            }
-          }
-          dst_s[b * TC_ROWS + el] = dst;
-        }
 
         // ---- epilogue 1: y = relu(fc1) -> bf16 operand (bias and one-hot columns are inside the GEMM) ----
         mbar_wait(&B->fc1d, par, abortf);
@@ -525,6 +503,60 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&B->yready);
+
+        // ---- while the y-side gate products run: everything that does not depend on the network.
+        //      Availability mask, the epsilon draw (it depends on the mask, not on Q), the environment's
+        //      reward/done and record address, and the requests for the next step's bytes. ----
+        uint32_t mask = 0;
+        int pick = -1;
+        float reward = 0.f;
+        int done = 0;
+        if (half == 0) {
+          const float eps = eps_at(p, t);
+          if (is_row) {
+            uint8_t* avd = rec + p.rl.off_avail + ai * A;
+            if (L.avail_bulk) {
+              mbar_wait(&B->full[b], (it >> 1) & 1, abortf);  // completed long ago; orders the bulk-written bytes
+#pragma unroll
+              for (int a = 0; a < 32; ++a)
+                if (a < A) mask |= (avd[a] ? 1u : 0u) << a;
+            } else {
+#pragma unroll
+              for (int a = 0; a < 32; ++a)
+                if (a < A) {
+                  asm volatile("" : "+r"(av_raw[a]));  // keeps the byte's use here, a whole step after its load
+                  mask |= (av_raw[a] ? 1u : 0u) << a;
+                  avd[a] = (uint8_t)av_raw[a];
+                }
+              if (s + 1 < p.T) {
+                const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
+#pragma unroll
+                for (int a = 0; a < 32; ++a)
+                  if (a < A) av_raw[a] = av[a];
+              }
+            }
+            if (mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)e, (uint32_t)ai);
+          }
+          if (is_env) {
+            asm volatile("" : "+f"(reward_raw), "+r"(done_raw));
+            reward = reward_raw;
+            done = done_raw ? 1 : 0;
+            if (s + 1 < p.T) {
+              reward_raw = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
+              done_raw = p.done[(size_t)(s + 1) * p.env_step_stride + e];
+            }
+            unsigned long long dst = 0;
+            if (ok) {
+              dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
+              if (pos == 0) {  // an episode opens in this slot
+                p.slot_epid[slot] = epc * (long long)p.E + e;
+                p.slot_len[slot] = 0;
+                p.slot_complete[slot] = 0;
+              }
+            }
+            dst_s[b * TC_ROWS + el] = dst;
+          }
+        }
 
         // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand.
         //      The r and z accumulators hold half the pre-activation: sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 ----
@@ -561,36 +593,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 
         // ---- epilogue 3: half 0 chooses and records; half 1 prepares the next step's operand ----
         if (half == 0) {
-          // the random branch does not depend on Q: drawn while fc2 runs
-          int pick = -1;
-          if (is_row && mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)e, (uint32_t)ai);
           mbar_wait(&B->fc2d, par, abortf);
           tc_fence_after_sync();
-          uint32_t qlo[16], qhi[16];
-          tmem_ld16(tmem + lane_addr + TM_Q, qlo);
-          if (L.NQ == 32) {
-            tmem_ld16(tmem + lane_addr + TM_Q + 16, qhi);
-          } else {
-#pragma unroll
-            for (int a = 0; a < 16; ++a) qhi[a] = 0;
-          }
+          uint32_t qv[NQ];
+          tmem_ld16(tmem + lane_addr + TM_Q, *reinterpret_cast<uint32_t(*)[16]>(qv));
+          if (NQ == 32) tmem_ld16(tmem + lane_addr + TM_Q + 16, *reinterpret_cast<uint32_t(*)[16]>(qv + NQ - 16));
           tmem_ld_wait();
           tc_fence_before_sync();
           if (is_row) {
-            // greedy rule on registers: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr
+            // greedy rule on registers: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr.
+            // Unavailable (and padding) entries become -inf; NaN never compares greater or equal.
+            float qm[NQ];
             float m = -INFINITY;
 #pragma unroll
-            for (int a = 0; a < 32; ++a) {
-              const float qa = __uint_as_float(a < 16 ? qlo[a & 15] : qhi[a & 15]);
-              if (a < L.NQ && ((mask >> a) & 1u) && qa > m) m = qa;
+            for (int a = 0; a < NQ; ++a) {
+              qm[a] = ((mask >> a) & 1u) ? __uint_as_float(qv[a]) : -INFINITY;
+              if (qm[a] > m) m = qm[a];
             }
             const float thr = __fsub_rn(m, 1e-4f);
             int g = __ffs(mask) - 1;
 #pragma unroll
-            for (int a = 31; a >= 0; --a) {
-              const float qa = __uint_as_float(a < 16 ? qlo[a & 15] : qhi[a & 15]);
-              if (a < L.NQ && ((mask >> a) & 1u) && qa >= thr) g = a;
-            }
+            for (int a = NQ - 1; a >= 0; --a)
+              if (((mask >> a) & 1u) && qm[a] >= thr) g = a;
             const int act = mask == 0 ? 0 : (pick >= 0 ? pick : g);
             c_steps += 1;
             c_explore += pick >= 0 ? 1u : 0u;
@@ -601,17 +625,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               la = act;
             }
             float* qrow = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
+            if ((A & 1) == 0) {  // rows of an even number of floats start on 8-byte boundaries
 #pragma unroll
-            for (int a = 0; a < 16; ++a)
-              if (a < A) qrow[a] = __uint_as_float(qlo[a]);
+              for (int a = 0; a < NQ; a += 2)
+                if (a < A) *reinterpret_cast<float2*>(qrow + a) = make_float2(__uint_as_float(qv[a]), __uint_as_float(qv[a + 1]));
+            } else {
 #pragma unroll
-            for (int a = 0; a < 16; ++a)
-              if (16 + a < A) qrow[16 + a] = __uint_as_float(qhi[a]);
+              for (int a = 0; a < NQ; ++a)
+                if (a < A) qrow[a] = __uint_as_float(qv[a]);
+            }
             reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
-            uint8_t* avd = rec + p.rl.off_avail + ai * A;
-#pragma unroll
-            for (int a = 0; a < 32; ++a)
-              if (a < A) avd[a] = (uint8_t)((mask >> a) & 1u);
             const int tk = p.trace_first + s;
             if (tk < p.trace_cap) {
               const size_t trow = ((size_t)tk * p.E + e) * n + ai;
@@ -696,17 +719,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 
 // Returns the number of kernels launched or a negative cudaError.
 int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream) {
-  const TcLayout L = tc_layout(p.n, p.D, p.A, (int)p.rl.rec_bytes);
+  TcLayout L = tc_layout(p.n, p.D, p.A, (int)p.rl.rec_bytes);
   if (reinterpret_cast<uintptr_t>(p.obs) % 16) return -(int)cudaErrorMisalignedAddress;
-  static uint32_t configured = 0;
-  if (L.total > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(actor_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+  // availability bytes ride with the observation copies when every environment's block is 16-byte sized and
+  // aligned; otherwise the row threads fetch them one step ahead
+  L.avail_bulk = ((p.n * p.A) % 16 == 0 && reinterpret_cast<uintptr_t>(p.avail) % 16 == 0) ? 1 : 0;
+  auto kernel = L.NQ == 16 ? actor_tc_kernel<16> : actor_tc_kernel<32>;
+  static uint32_t configured[2] = {0, 0};
+  uint32_t& conf = configured[L.NQ == 16 ? 0 : 1];
+  if (L.total > conf) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return -(int)e;
-    configured = L.total;
+    conf = L.total;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;
-  actor_tc_kernel<<<grid, TC_THREADS, L.total, stream>>>(p, L);
+  kernel<<<grid, TC_THREADS, L.total, stream>>>(p, L);
   const cudaError_t err = cudaGetLastError();
   return err == cudaSuccess ? 1 : -(int)err;
 }
