@@ -51,7 +51,7 @@ struct TcLayout {
   // packed weight image (same offsets in global and shared memory)
   uint32_t off_W1, off_Wih, off_Bin, off_Whh, off_W2, wbytes;
   // shared memory only
-  uint32_t off_xy, off_hb, off_oh, off_rec, off_dst, off_reset, off_rowoff, off_bar, total;
+  uint32_t off_xy, off_hb, off_oh, off_rec, off_dst, off_reset, off_rowoff, off_sel, off_bar, total;
 };
 
 // Operand K-columns beyond the data columns ("extension"): the fp32 biases and the two one-hot parts of
@@ -89,6 +89,7 @@ static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
   L.off_dst = o; o += 2u * TC_ROWS * 8;
   L.off_reset = o; o += TC_ROWS * 4;
   L.off_rowoff = o; o += TC_ROWS * 4;
+  L.off_sel = o; o += TC_ROWS * 8;
   L.off_bar = o; o += 128;
   L.total = o;
   return L;
@@ -187,7 +188,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 struct TcBars {
-  uint64_t full[2], xready, fc1d, yready, grud, hready, fc2d, stepd, wload;
+  uint64_t full[2], xready, fc1d, yready, grud, hready, fc2d, stepd, wload, selready;
   uint32_t tmem_base, abort;
 };
 
@@ -204,6 +205,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   unsigned long long* dst_s = reinterpret_cast<unsigned long long*>(smem + L.off_dst);  // [2][128]
   int32_t* reset_s = reinterpret_cast<int32_t*>(smem + L.off_reset);
   uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(smem + L.off_rowoff);
+  uint2* sel_s = reinterpret_cast<uint2*>(smem + L.off_sel);  // per row: availability mask, random pick or -1
   volatile uint32_t* abortf = &B->abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -222,6 +224,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     mbar_init(&B->fc2d, 1);
     mbar_init(&B->stepd, 256);
     mbar_init(&B->wload, 1);
+    mbar_init(&B->selready, 64);
     B->abort = 0;
     mbar_init_fence();
   }
@@ -360,6 +363,40 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       }
     }
     bulk_wait_all();
+   } else if (L.avail_bulk) {
+    // =========================== draw warps: availability mask and epsilon draw of every row ==============
+    // Neither depends on the network, so two otherwise idle warps prepare them at the start of each step
+    // from the availability bytes that arrived with the observations; epilogue 3 only reads the result.
+    const int r0 = tid - 10 * 32;  // 0..63, rows r0 and r0 + 64
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const int e0 = tile * L.ept;
+      const int R = min(L.ept, p.E - e0) * n;
+      for (int s = 0; s < p.T; ++s) {
+        const uint32_t b = it & 1;
+        mbar_wait(&B->stepd, sd & 1, abortf);  // prologue or previous step: the hand-off array is free again
+        ++sd;
+        mbar_wait(&B->full[b], (it >> 1) & 1, abortf);
+        const uint32_t t = p.t0 + (uint32_t)s;
+        const float eps = eps_at(p, t);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int r = r0 + 64 * u;
+          if (r < R) {
+            const int rel = r / n, rai = r - rel * n;
+            const uint8_t* avd = recs + b * buf_bytes + (uint32_t)rel * rec_bytes + p.rl.off_avail + rai * A;
+            uint32_t mask = 0;
+            for (int a = 0; a < A; ++a) mask |= (avd[a] ? 1u : 0u) << a;
+            int pick = -1;
+            if (mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)(e0 + rel), (uint32_t)rai);
+            sel_s[r] = make_uint2(mask, (uint32_t)pick);
+          }
+        }
+        mbar_arrive(&B->selready);
+        ++it;
+      }
+      mbar_wait(&B->stepd, sd & 1, abortf);  // last step of the tile
+      ++sd;
+    }
    }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(TC_REGS_EPILOGUE));
@@ -415,7 +452,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const int R = ne * n;
       const bool live = row < R;
       const bool is_row = live && half == 0;             // owner of the row's choice
-      const bool is_env = is_row && ai == 0;             // owner of the environment's cursor
+      const bool is_env = live && half == 1 && ai == 0;  // owner of the environment's cursor (half 1 has slack)
       const int e = e0 + el;
       const size_t grow = (size_t)e * n + ai;             // global row
       int32_t slot = 0, pos = 0, ok = 0, la = -1;
@@ -504,58 +541,49 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         tc_fence_before_sync();
         mbar_arrive(&B->yready);
 
-        // ---- while the y-side gate products run: everything that does not depend on the network.
-        //      Availability mask, the epsilon draw (it depends on the mask, not on Q), the environment's
-        //      reward/done and record address, and the requests for the next step's bytes. ----
+        // ---- while the y-side gate products run: work that does not depend on the network - the environment's
+        //      reward/done, record address and the requests for the next step's values ----
         uint32_t mask = 0;
         int pick = -1;
         float reward = 0.f;
         int done = 0;
-        if (half == 0) {
+        if (is_row && !L.avail_bulk) {
+          // availability bytes fetched by this thread one step ahead (shapes whose rows cannot be bulk-copied)
           const float eps = eps_at(p, t);
-          if (is_row) {
-            uint8_t* avd = rec + p.rl.off_avail + ai * A;
-            if (L.avail_bulk) {
-              mbar_wait(&B->full[b], (it >> 1) & 1, abortf);  // completed long ago; orders the bulk-written bytes
+          uint8_t* avd = rec + p.rl.off_avail + ai * A;
 #pragma unroll
-              for (int a = 0; a < 32; ++a)
-                if (a < A) mask |= (avd[a] ? 1u : 0u) << a;
-            } else {
-#pragma unroll
-              for (int a = 0; a < 32; ++a)
-                if (a < A) {
-                  asm volatile("" : "+r"(av_raw[a]));  // keeps the byte's use here, a whole step after its load
-                  mask |= (av_raw[a] ? 1u : 0u) << a;
-                  avd[a] = (uint8_t)av_raw[a];
-                }
-              if (s + 1 < p.T) {
-                const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
-#pragma unroll
-                for (int a = 0; a < 32; ++a)
-                  if (a < A) av_raw[a] = av[a];
-              }
+          for (int a = 0; a < 32; ++a)
+            if (a < A) {
+              asm volatile("" : "+r"(av_raw[a]));  // keeps the byte's use here, a whole step after its load
+              mask |= (av_raw[a] ? 1u : 0u) << a;
+              avd[a] = (uint8_t)av_raw[a];
             }
-            if (mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)e, (uint32_t)ai);
+          if (s + 1 < p.T) {
+            const uint8_t* av = p.avail + (size_t)(s + 1) * p.avail_step_stride + grow * A;
+#pragma unroll
+            for (int a = 0; a < 32; ++a)
+              if (a < A) av_raw[a] = av[a];
           }
-          if (is_env) {
-            asm volatile("" : "+f"(reward_raw), "+r"(done_raw));
-            reward = reward_raw;
-            done = done_raw ? 1 : 0;
-            if (s + 1 < p.T) {
-              reward_raw = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
-              done_raw = p.done[(size_t)(s + 1) * p.env_step_stride + e];
-            }
-            unsigned long long dst = 0;
-            if (ok) {
-              dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
-              if (pos == 0) {  // an episode opens in this slot
-                p.slot_epid[slot] = epc * (long long)p.E + e;
-                p.slot_len[slot] = 0;
-                p.slot_complete[slot] = 0;
-              }
-            }
-            dst_s[b * TC_ROWS + el] = dst;
+          if (mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)e, (uint32_t)ai);
+        }
+        if (is_env) {
+          asm volatile("" : "+f"(reward_raw), "+r"(done_raw));
+          reward = reward_raw;
+          done = done_raw ? 1 : 0;
+          if (s + 1 < p.T) {
+            reward_raw = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
+            done_raw = p.done[(size_t)(s + 1) * p.env_step_stride + e];
           }
+          unsigned long long dst = 0;
+          if (ok) {
+            dst = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
+            if (pos == 0) {  // an episode opens in this slot
+              p.slot_epid[slot] = epc * (long long)p.E + e;
+              p.slot_len[slot] = 0;
+              p.slot_complete[slot] = 0;
+            }
+          }
+          dst_s[b * TC_ROWS + el] = dst;
         }
 
         // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand.
@@ -600,6 +628,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           if (NQ == 32) tmem_ld16(tmem + lane_addr + TM_Q + 16, *reinterpret_cast<uint32_t(*)[16]>(qv + NQ - 16));
           tmem_ld_wait();
           tc_fence_before_sync();
+          if (is_row && L.avail_bulk) {
+            mbar_wait(&B->selready, par, abortf);
+            const uint2 sp = sel_s[row];
+            mask = sp.x;
+            pick = (int)sp.y;
+          }
           if (is_row) {
             // greedy rule on registers: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr.
             // Unavailable (and padding) entries become -inf; NaN never compares greater or equal.
@@ -644,6 +678,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             }
             if (p.actions_out && s == p.T - 1) p.actions_out[grow] = act;
           }
+        } else {
           if (is_env) {
             int closed = 0;
             if (ok) {
@@ -664,11 +699,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             }
             reset_s[el] = closed;
           }
-        } else if (s + 1 < p.T) {
-          mbar_wait(&B->full[b ^ 1], ((it + 1) >> 1) & 1, abortf);
-          convert_x(b ^ 1, R);
-          fence_proxy_async_smem();
-          mbar_arrive(&B->xready);
+          if (s + 1 < p.T) {
+            mbar_wait(&B->full[b ^ 1], ((it + 1) >> 1) & 1, abortf);
+            convert_x(b ^ 1, R);
+            fence_proxy_async_smem();
+            mbar_arrive(&B->xready);
+          }
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         // ---- a closed episode restarts from a zero hidden state and no last action ----
