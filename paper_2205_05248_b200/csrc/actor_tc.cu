@@ -637,18 +637,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           if (is_row) {
             // greedy rule on registers: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr.
             // Unavailable (and padding) entries become -inf; NaN never compares greater or equal.
+            // Written as independent operations and a reduction tree: one thread, so instruction-level
+            // parallelism is all there is.  fmaxf ignores a NaN operand, like the "greater than" scan it replaces.
             float qm[NQ];
-            float m = -INFINITY;
 #pragma unroll
-            for (int a = 0; a < NQ; ++a) {
-              qm[a] = ((mask >> a) & 1u) ? __uint_as_float(qv[a]) : -INFINITY;
-              if (qm[a] > m) m = qm[a];
-            }
-            const float thr = __fsub_rn(m, 1e-4f);
-            int g = __ffs(mask) - 1;
+            for (int a = 0; a < NQ; ++a) qm[a] = ((mask >> a) & 1u) ? __uint_as_float(qv[a]) : -INFINITY;
+            float red[NQ];
 #pragma unroll
-            for (int a = NQ - 1; a >= 0; --a)
-              if (((mask >> a) & 1u) && qm[a] >= thr) g = a;
+            for (int a = 0; a < NQ; ++a) red[a] = qm[a];
+#pragma unroll
+            for (int w = NQ / 2; w >= 1; w >>= 1)
+#pragma unroll
+              for (int a = 0; a < w; ++a) red[a] = fmaxf(red[a], red[a + w]);
+            const float thr = __fsub_rn(red[0], 1e-4f);
+            uint32_t ge = 0;
+#pragma unroll
+            for (int a = 0; a < NQ; ++a) ge |= (qm[a] >= thr ? 1u : 0u) << a;
+            ge &= mask;
+            const int g = ge ? __ffs(ge) - 1 : __ffs(mask) - 1;
             const int act = mask == 0 ? 0 : (pick >= 0 ? pick : g);
             c_steps += 1;
             c_explore += pick >= 0 ? 1u : 0u;
