@@ -66,6 +66,30 @@ def flops_per_agent_step(cfg: dict) -> float:
     return 2.0 * H * (D + 6 * H + A) + 25.0 * H
 
 
+def measured_traffic(kernel_name: str, agent_steps_per_launch: float):
+    """DRAM bytes per launch from the committed ncu record of this kernel, or None if there is no record or the
+    kernel sources have changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", f"{kernel_name}_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    rec = {}
+    for line in open(path):
+        if line.startswith("#") or ":" not in line:
+            continue
+        k, v = line.split(":", 1)
+        rec[k.strip()] = v.strip()
+    try:
+        h = hashlib.sha256()
+        for f in rec["source_files"].split():
+            h.update(open(os.path.join(ROOT, f), "rb").read())
+        if h.hexdigest() != rec["source_sha256"]:
+            return None
+        return float(rec["dram_bytes_per_agent_step"]) * agent_steps_per_launch
+    except (KeyError, OSError, ValueError):
+        return None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -136,7 +160,8 @@ def dist_setup(n_gpus: int):
     if world > 1:
         import torch
         import torch.distributed as dist
-        torch.cuda.set_device(local)
+        if torch.cuda.is_available():
+            torch.cuda.set_device(local)
         dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
     return rank, world, local
 
@@ -273,9 +298,10 @@ def main():
     bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T) * E * n * T
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     flop_rate = flops_per_agent_step(cfg) * E * n * T / (kernel_ms * 1e-3) / 1e12
+    kname = "actor_%s_kernel" % ("tc" if actor.kernel_name == "tcgen05" else "ffma")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
-                "kernel": "actor_%s_kernel" % ("tc" if actor.kernel_name == "tcgen05" else "ffma"),
+                "frac": achieved / peaks["hbm_gbs"], "traffic": measured_traffic(kname, E * n * T),
+                "peak_source": peak_kind, "kernel": kname,
                 "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T),
                 "tflops_effective": flop_rate}
 
