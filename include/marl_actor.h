@@ -58,6 +58,8 @@ extern "C" {
 #define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
 #define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
 #define MARL_STATUS_BAD_INDEX 4u /* a ring or state index was out of range and the access was skipped */
+/* Bits 8 and above of the status word carry a diagnostic code when MARL_STATUS_TIMEOUT is set (which wait of
+ * which warp expired first); they have no meaning otherwise. */
 
 typedef struct marl_actor marl_actor_t; /* opaque; owned by the library; freed by marl_actor_destroy */
 
@@ -246,6 +248,13 @@ int marl_actor_reset(marl_actor_t* a);
 
 /* SYNCHRONISES the stream and frees what the library allocated. */
 void marl_actor_destroy(marl_actor_t* a);
+
+/* Failure-detection self-test (no counterpart in the paper): launches a one-block kernel that waits, with the
+ * bounded wait the tensor-core kernel uses for all of its hand-offs, on a barrier that nothing completes.  The
+ * wait gives up after poll_limit polls (1 .. 1000000; 20000 is a few tens of milliseconds) and the kernel
+ * reports it.  SYNCHRONISES the stream.  *status_out (host) receives MARL_STATUS_TIMEOUT | 0x100 when the
+ * mechanism works.  The CUDA context stays usable afterwards. */
+int marl_selftest_bounded_wait(void* stream, uint32_t poll_limit, uint32_t* status_out);
 
 /* Name of the step kernel in use: "ffma" or "tcgen05". */
 const char* marl_actor_kernel_name(const marl_actor_t* a);

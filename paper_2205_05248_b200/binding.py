@@ -26,7 +26,7 @@ EXPORTS = [
     "marl_actor_step", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
     "marl_actor_set_trace", "marl_ring_view", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
-    "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc",
+    "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc", "marl_selftest_bounded_wait",
 ]
 
 
@@ -103,6 +103,7 @@ def load_library():
         lib.marl_rollout_staged.argtypes = [P, P, P, P, P, C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout_noalloc.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
+        lib.marl_selftest_bounded_wait.argtypes = [P, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.marl_actor_set_trace.argtypes = [P, P, P, C.c_int32]
         lib.marl_ring_view.argtypes = [P, C.POINTER(RingView)]
         lib.marl_actor_get_state.argtypes = [P, C.POINTER(StateView)]
@@ -139,6 +140,14 @@ def marl_actor_query_sizes(cfg: dict) -> dict:
     c = make_config(cfg)
     _check(load_library().marl_actor_query_sizes(C.byref(c), C.byref(s)))
     return {k: getattr(s, k) for k, _ in Sizes._fields_}
+
+
+def marl_selftest_bounded_wait(poll_limit: int = 20000) -> int:
+    """Runs the bounded-wait self-test on the current stream; returns the reported status word."""
+    st = C.c_uint32(0)
+    stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().marl_selftest_bounded_wait(C.c_void_p(stream), C.c_uint32(poll_limit), C.byref(st)))
+    return int(st.value)
 
 
 def _dptr(t):

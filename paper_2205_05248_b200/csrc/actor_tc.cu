@@ -755,7 +755,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (tid == 0 && B->abort) atomicOr(p.status, MARL_STATUS_TIMEOUT);
+  if (tid == 0 && B->abort) {
+    atomicOr(p.status, MARL_STATUS_TIMEOUT);
+    // diagnosis: which barrier (index inside the barrier block) and which warp gave up first
+    atomicCAS(p.status + 1, 0u, ((((B->abort & 0xFFFFFu) - (smem_u32(B) & 0xFFFFFu)) >> 3) & 0xFFu) | (((B->abort >> 20) & 0xFFu) << 8));
+  }
   if (warp == 8) tmem_dealloc(tmem, TM_COLS);
 }
 

@@ -198,7 +198,7 @@ __global__ void init_state_kernel(int E, int n, int H, int S, int C, float* h, i
     complete[i] = 0;
   }
   if (i0 < CNT_N) counters[i0] = 0;
-  if (i0 == 0) *status = 0;
+  if (i0 < 4) status[i0] = 0;
 }
 
 static int enqueue_reset(marl_actor* a) {
@@ -607,11 +607,11 @@ int marl_actor_set_state(marl_actor_t* a, const marl_state_view_t* in) {
 int marl_actor_status(marl_actor_t* a, uint32_t* device_status, marl_counters_t* counters) {
   if (!a) return fail(MARL_EINVAL, "actor is NULL");
   uint64_t cnt[CNT_N];
-  uint32_t st = 0;
+  uint32_t st[4] = {0, 0, 0, 0};
   CU_TRY(cudaMemcpyAsync(cnt, a->state + a->so.counters, sizeof(cnt), cudaMemcpyDeviceToHost, a->stream));
-  CU_TRY(cudaMemcpyAsync(&st, a->state + a->so.status, sizeof(st), cudaMemcpyDeviceToHost, a->stream));
+  CU_TRY(cudaMemcpyAsync(st, a->state + a->so.status, sizeof(st), cudaMemcpyDeviceToHost, a->stream));
   CU_TRY(cudaStreamSynchronize(a->stream));
-  if (device_status) *device_status = st;
+  if (device_status) *device_status = st[0] | (st[1] << 8);  // bits 8..: timeout diagnosis (barrier, warp)
   if (counters) {
     counters->agent_steps = cnt[CNT_AGENT_STEPS];
     counters->episodes = cnt[CNT_EPISODES];

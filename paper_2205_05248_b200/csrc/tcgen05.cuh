@@ -47,17 +47,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after `limit` polls (each poll may itself block for a hardware-defined time),
+// Bounded wait: gives up after `limit` polls (each poll may itself block for a hardware-defined time; the
+// default is about a second),
 // raises *abort_flag (shared) so that every later wait in the block returns at once, and reports failure.
-// A kernel that saw a failure finishes its loops on garbage values but keeps every index in range.
+// The flag keeps the first failure's code: the barrier's byte offset in shared memory (low 20 bits) and the
+// waiting warp (bits 20..27), for diagnosis.  A kernel that saw a failure finishes its loops on garbage values
+// but keeps every index in range.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t limit = 4000000u) {
+                                          uint32_t limit = 300000u) {
   for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (i > 64) __nanosleep(32);
   }
-  *abort_flag = 1;
+  atomicCAS(const_cast<uint32_t*>(abort_flag), 0u, (smem_u32(bar) & 0xFFFFFu) | ((threadIdx.x >> 5) << 20) | 0x80000000u);
   return false;
 }
 

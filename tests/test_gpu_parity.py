@@ -244,3 +244,17 @@ def test_host_errors_are_codes_not_crashes():
     actor.destroy()
     with pytest.raises(binding.MarlError, match="tensor-core"):
         binding.Actor(dict(cfg, precision="fp32"), kernel="tensor")
+
+
+def test_bounded_wait_gives_up_and_context_survives():
+    """A device-side wait on a barrier that nothing completes expires, reports TIMEOUT through the status word
+    and leaves the context usable (no trap, no hang): the failure path of every hand-off in the tcgen05 kernel."""
+    st = binding.marl_selftest_bounded_wait(20000)
+    assert st & binding.STATUS_TIMEOUT and st & 0x100
+    x = torch.arange(8, device="cuda").sum().item()      # the context still works
+    assert x == 28
+    cfg = workloads.small_config(H=64, D=8, precision="bf16", E=40, C=40)
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w, kernel="tensor")
+    assert actor.status()[0] == 0                        # and a real rollout afterwards is clean
+    actor.destroy()
