@@ -40,6 +40,7 @@ constexpr int TC_THREADS = 384;  // two epilogue warpgroups + one service warpgr
 // (384 * 168 = 64512); the service warpgroup drops to 88 and each epilogue warpgroup rises to 208:
 // 256 * 208 + 128 * 88 = 64512, exactly the launch total.
 constexpr int TC_REGS_EPILOGUE = 208, TC_REGS_SERVICE = 88;
+constexpr int TC_TAB = 68;                 // row stride (floats) of the last-action table: conflict-free float4 rows
 constexpr uint32_t TC_LBO_A = 2048;        // k-chunk stride of a 128-row operand
 constexpr uint32_t TC_LBO_X = 2048 + 16;   // padded for the observation operand: spreads the converter's stores
 constexpr uint32_t TC_SMEM_MAX = 232448;   // 227 KB opt-in limit per block
@@ -49,18 +50,21 @@ constexpr uint32_t TM_FC1 = 0, TM_R = 64, TM_Z = 128, TM_IN = 192, TM_HN = 256, 
 struct TcLayout {
   int32_t Dk, NQ, nchunk, ept, ohK, ohc, avail_bulk, pad_;
   // packed weight image (same offsets in global and shared memory)
-  uint32_t off_W1, off_Wih, off_Bin, off_Whh, off_W2, wbytes;
+  uint32_t off_W1, off_Wih, off_Whh, off_Bg, off_Bhn, off_W2, off_tab_la, wbytes;
   // shared memory only
-  uint32_t off_xy, off_hb, off_oh, off_rec, off_dst, off_reset, off_rowoff, off_sel, off_bar, total;
+  uint32_t off_xy, off_hb, off_oh, off_rec, off_dst, off_reset, off_la, off_rowoff, off_sel, off_bar, total;
 };
 
 // Operand K-columns beyond the data columns ("extension"): the fp32 biases and the two one-hot parts of
 // the network input enter the GEMMs as extra K columns, so the epilogues add nothing.
-//   one-hot operand tile (A side, per row):  col 0..2 = 1, col 3+i = [agent == i], col 3+n+a = [last action == a]
+//   one-hot operand tile (A side, per row, constant for a tile):  col 0..2 = 1, col 3+i = [agent == i]
 //   fc1 weights (B side):    k = Dk+0..2: b1 split into three bf16 pieces (their sum is b1 to fp32 accuracy),
-//                            k = Dk+3+i: W1[:, D+i],  k = Dk+3+n+a: W1[:, D+n+a]
-//   W_hh, W2, and a small tile for the candidate gate's input bias: bias pieces at k = 64..66 (resp. 0..2),
-//   multiplied by the three ones of the one-hot tile; all other extension entries are zero.
+//                            k = Dk+3+i: W1[:, D+i]
+//   gate-bias tile, candidate-hidden-bias tile and W2: bias pieces at k = 0..2 (resp. 64..66), multiplied by
+//   the three ones of the one-hot tile; all other extension entries are zero.
+// The last-action one-hot is the only input that depends on the previous step's choice; keeping it out of the
+// GEMM lets fc1 of step s+1 run entirely during step s.  Its term W1[:, D+n+last] is added in epilogue 1 from
+// a small fp32 table.
 // The reset and update rows of W_ih / W_hh and their biases are stored halved (exact in bf16), so that
 // sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 needs no multiply in the epilogue.
 static uint32_t up16(uint32_t v) { return (v + 15u) & ~15u; }
@@ -72,14 +76,16 @@ static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
   L.NQ = A <= 16 ? 16 : 32;
   L.nchunk = L.Dk / 8;
   L.ept = TC_ROWS / n;
-  L.ohK = (3 + n + A + 15) & ~15;
+  L.ohK = (3 + n + 15) & ~15;
   L.ohc = L.ohK / 8;
   uint32_t o = 0;
   L.off_W1 = o; o += (uint32_t)(L.nchunk + L.ohc) * TC_H * 16;
   L.off_Wih = o; o += 8u * 3 * TC_H * 16;
-  L.off_Bin = o; o += 2u * TC_H * 16;
-  L.off_Whh = o; o += 10u * 3 * TC_H * 16;
+  L.off_Whh = o; o += 8u * 3 * TC_H * 16;
+  L.off_Bg = o; o += 2u * 3 * TC_H * 16;   // gate biases: r, z (both sides summed, halved) and the candidate's input bias
+  L.off_Bhn = o; o += 2u * TC_H * 16;      // the candidate's hidden bias
   L.off_W2 = o; o += 10u * L.NQ * 16;
+  L.off_tab_la = o; o += up16(sizeof(float) * A * TC_TAB);  // W1[:, D+n+a] as fp32 rows: the last-action term
   L.wbytes = o;
   const uint32_t xbytes = (uint32_t)L.nchunk * TC_LBO_X;
   L.off_xy = o; o += up16(xbytes > 8 * TC_LBO_A ? xbytes : 8 * TC_LBO_A);
@@ -88,6 +94,7 @@ static TcLayout tc_layout(int n, int D, int A, int rec_bytes) {
   L.off_rec = o; o += 2u * L.ept * (uint32_t)rec_bytes;
   L.off_dst = o; o += 2u * TC_ROWS * 8;
   L.off_reset = o; o += TC_ROWS * 4;
+  L.off_la = o; o += TC_ROWS * 4;
   L.off_rowoff = o; o += TC_ROWS * 4;
   L.off_sel = o; o += TC_ROWS * 8;
   L.off_bar = o; o += 128;
@@ -149,7 +156,7 @@ void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b
   for (int j = 0; j < H; ++j) {
     for (int k = 0; k < D; ++k) put(L.off_W1, H, j, k, W1[(size_t)j * I + k]);
     put3(L.off_W1, H, j, L.Dk, b1[j]);
-    for (int i = 0; i < n + A; ++i) put(L.off_W1, H, j, L.Dk + 3 + i, W1[(size_t)j * I + D + i]);
+    for (int i = 0; i < n; ++i) put(L.off_W1, H, j, L.Dk + 3 + i, W1[(size_t)j * I + D + i]);
   }
   for (int r = 0; r < 3 * H; ++r) {
     const float sc = r < 2 * H ? 0.5f : 1.0f;  // reset and update rows are stored halved
@@ -158,16 +165,19 @@ void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b
       put(L.off_Whh, 3 * H, r, k, sc * bf16_value(Whh[(size_t)r * H + k]));
     }
     if (r < 2 * H) {
-      put3(L.off_Whh, 3 * H, r, H, 0.5f * (bih[r] + bhh[r]));
+      put3(L.off_Bg, 3 * H, r, 0, 0.5f * (bih[r] + bhh[r]));
     } else {
-      put3(L.off_Whh, 3 * H, r, H, bhh[r]);
-      put3(L.off_Bin, H, r - 2 * H, 0, bih[r]);
+      put3(L.off_Bg, 3 * H, r, 0, bih[r]);
+      put3(L.off_Bhn, H, r - 2 * H, 0, bhh[r]);
     }
   }
   for (int a = 0; a < A; ++a) {
     for (int k = 0; k < H; ++k) put(L.off_W2, L.NQ, a, k, W2[(size_t)a * H + k]);
     put3(L.off_W2, L.NQ, a, H, b2[a]);
   }
+  float* tla = reinterpret_cast<float*>(o + L.off_tab_la);
+  for (int a = 0; a < A; ++a)
+    for (int j = 0; j < H; ++j) tla[a * TC_TAB + j] = bf16_value(W1[(size_t)j * I + D + n + a]);
 }
 
 void tc_tiling(int E, int n, int /*sms*/, int* ept, int* num_tiles) {
@@ -204,6 +214,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   uint8_t* recs = smem + L.off_rec;
   unsigned long long* dst_s = reinterpret_cast<unsigned long long*>(smem + L.off_dst);  // [2][128]
   int32_t* reset_s = reinterpret_cast<int32_t*>(smem + L.off_reset);
+  int32_t* la_s = reinterpret_cast<int32_t*>(smem + L.off_la);    // last action of every row, for the half-1 threads
+  const float* tab_la = reinterpret_cast<const float*>(smem + L.off_tab_la);
   uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(smem + L.off_rowoff);
   uint2* sel_s = reinterpret_cast<uint2*>(smem + L.off_sel);  // per row: availability mask, random pick or -1
   volatile uint32_t* abortf = &B->abort;
@@ -250,7 +262,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(TC_REGS_SERVICE));
    if (warp == 8) {
     // =========================== MMA warp: lane 0 issues every tcgen05.mma ===========================
-    const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, NQ);
+    const uint32_t id64 = idesc_bf16_f32(128, 64), id128 = idesc_bf16_f32(128, 128), idq = idesc_bf16_f32(128, NQ), id192 = idesc_bf16_f32(128, 192);
     const uint32_t lbo_w1 = TC_H * 16, lbo_g = 3 * TC_H * 16, lbo_q = (uint32_t)NQ * 16;
     const uint32_t gate_n = 2 * TC_H * 16;  // byte offset of the candidate-gate rows inside a k-chunk of W_ih / W_hh
     // descriptors of the first k-step of every operand; a later k-step adds (2 * LBO) >> 4 to the address field
@@ -259,53 +271,50 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     const uint64_t d_W1 = smem_desc(smem_u32(smem + L.off_W1), lbo_w1, 128);
     const uint64_t d_W1oh = smem_desc(smem_u32(smem + L.off_W1) + (uint32_t)L.nchunk * lbo_w1, lbo_w1, 128);
     const uint64_t d_Wih = smem_desc(smem_u32(smem + L.off_Wih), lbo_g, 128);
-    const uint64_t d_Wih_n = smem_desc(smem_u32(smem + L.off_Wih) + gate_n, lbo_g, 128);
     const uint64_t d_Whh = smem_desc(smem_u32(smem + L.off_Whh), lbo_g, 128);
     const uint64_t d_Whh_n = smem_desc(smem_u32(smem + L.off_Whh) + gate_n, lbo_g, 128);
-    const uint64_t d_Bin = smem_desc(smem_u32(smem + L.off_Bin), lbo_w1, 128);
+    const uint64_t d_Bg = smem_desc(smem_u32(smem + L.off_Bg), lbo_g, 128);
+    const uint64_t d_Bhn = smem_desc(smem_u32(smem + L.off_Bhn), lbo_w1, 128);
     const uint64_t d_W2 = smem_desc(smem_u32(smem + L.off_W2), lbo_q, 128);
     const uint64_t k_x = (2 * TC_LBO_X) >> 4, k_a = (2 * TC_LBO_A) >> 4, k_w1 = (2 * lbo_w1) >> 4, k_g = (2 * lbo_g) >> 4,
                    k_q = (2 * lbo_q) >> 4;
     const int ks_obs = L.Dk / 16, ks_oh = L.ohK / 16;
-    // The observation columns of fc1 need only the converted observations, so they are issued as soon as
-    // those are ready - for step s+1 while step s is still in its third epilogue.  The one-hot / bias columns
-    // follow once the step before has published its actions.
-    auto issue_fc1_obs = [&]() {
+    // fc1 of a step depends only on the converted observations (the last-action term is added in epilogue 1),
+    // so it is issued as soon as those are ready - for step s+1 while step s is still in its third epilogue.
+    auto issue_fc1 = [&]() {
       mbar_wait(&B->xready, it & 1, abortf);
       tc_fence_after_sync();
-      if (lane == 0)
+      if (lane == 0) {
         for (int ks = 0; ks < ks_obs; ++ks) mma_bf16(tmem + TM_FC1, d_x + ks * k_x, d_W1 + ks * k_w1, id64, ks > 0);
+        for (int ks = 0; ks < ks_oh; ++ks) mma_bf16(tmem + TM_FC1, d_oh + ks * k_a, d_W1oh + ks * k_w1, id64, 1);
+        mma_commit(&B->fc1d);
+      }
       __syncwarp();
     };
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      issue_fc1_obs();
+      issue_fc1();
       for (int s = 0; s < p.T; ++s) {
         const uint32_t par = it & 1;
-        mbar_wait(&B->stepd, sd & 1, abortf);  // prologue or previous step: hidden and one-hot operands in place
+        mbar_wait(&B->stepd, sd & 1, abortf);  // prologue or previous step: hidden operand in place
         ++sd;
         tc_fence_after_sync();
         if (lane == 0) {
-          for (int ks = 0; ks < ks_oh; ++ks) mma_bf16(tmem + TM_FC1, d_oh + ks * k_a, d_W1oh + ks * k_w1, id64, 1);
-          mma_commit(&B->fc1d);
-          // h-side gate products and all gate biases: independent of this step's fc1, overlap epilogue 1
+          // h-side gate products; the first MMA seeds r | z | candidate-input with their biases (r, z and the
+          // candidate's input part are contiguous in tensor memory: one N = 192 accumulator)
+          mma_bf16(tmem + TM_R, d_oh, d_Bg, id192, 0);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            mma_bf16(tmem + TM_R, d_h + ks * k_a, d_Whh + ks * k_g, id128, ks > 0);
+            mma_bf16(tmem + TM_R, d_h + ks * k_a, d_Whh + ks * k_g, id128, 1);
             mma_bf16(tmem + TM_HN, d_h + ks * k_a, d_Whh_n + ks * k_g, id64, ks > 0);
           }
-          mma_bf16(tmem + TM_R, d_oh, d_Whh + 4 * k_g, id128, 1);
-          mma_bf16(tmem + TM_HN, d_oh, d_Whh_n + 4 * k_g, id64, 1);
+          mma_bf16(tmem + TM_HN, d_oh, d_Bhn, id64, 1);
         }
         __syncwarp();
         mbar_wait(&B->yready, par, abortf);
         tc_fence_after_sync();
         if (lane == 0) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            mma_bf16(tmem + TM_R, d_y + ks * k_a, d_Wih + ks * k_g, id128, 1);
-            mma_bf16(tmem + TM_IN, d_y + ks * k_a, d_Wih_n + ks * k_g, id64, ks > 0);
-          }
-          mma_bf16(tmem + TM_IN, d_oh, d_Bin, id64, 1);
+          for (int ks = 0; ks < 4; ++ks) mma_bf16(tmem + TM_R, d_y + ks * k_a, d_Wih + ks * k_g, id192, 1);
           mma_commit(&B->grud);
         }
         __syncwarp();
@@ -319,7 +328,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         }
         __syncwarp();
         ++it;
-        if (s + 1 < p.T) issue_fc1_obs();
+        if (s + 1 < p.T) issue_fc1();
       }
       mbar_wait(&B->stepd, sd & 1, abortf);  // last step of the tile
       ++sd;
@@ -477,6 +486,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         }
         if (half == 0) {
           reset_s[row] = 0;
+          la_s[row] = live ? p.last_action[grow] : -1;
           for (int c = 0; c < L.ohc; ++c)
             *reinterpret_cast<uint4*>(oh + (uint32_t)c * TC_LBO_A + (uint32_t)row * 16u) = make_uint4(0, 0, 0, 0);
         }
@@ -486,7 +496,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           *reinterpret_cast<uint16_t*>(oh_col(1)) = 0x3F80;
           *reinterpret_cast<uint16_t*>(oh_col(2)) = 0x3F80;
           *reinterpret_cast<uint16_t*>(oh_col(3 + ai)) = 0x3F80;
-          if (la >= 0 && la < A) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0x3F80;
+          if (la >= A) la = -1;
           if (!L.avail_bulk) {
             const uint8_t* av = p.avail + grow * A;
 #pragma unroll
@@ -519,22 +529,36 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const uint32_t t = p.t0 + (uint32_t)s;
         uint8_t* rec = recs + b * buf_bytes + (uint32_t)el * rec_bytes;  // this row's environment record
 
-        // ---- epilogue 1: y = relu(fc1) -> bf16 operand (bias and one-hot columns are inside the GEMM) ----
+        // ---- epilogue 1: y = relu(fc1 + W1[:, last action]) -> bf16 operand.  Bias and agent-id column are
+        //      inside the GEMM; fc1 itself finished during the previous step. ----
         mbar_wait(&B->fc1d, par, abortf);
         tc_fence_after_sync();
+        {
+          // both published before the previous step's closing barrier; an episode that just ended has no last action
+          int last = reset_s[el] ? -1 : la_s[row];
+          if (last >= A) last = -1;
+          const float* tl = tab_la + (last >= 0 ? last : 0) * TC_TAB + cb;
 #pragma unroll
-        for (int c16 = 0; c16 < 2; ++c16) {
-          uint32_t v[16];
-          tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
-          tmem_ld_wait();
+          for (int c16 = 0; c16 < 2; ++c16) {
+            uint32_t v[16];
+            tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
+            tmem_ld_wait();
+            float y[16];
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const uint32_t* w = v + 8 * cc;
-            const uint4 o = make_uint4(pack_bf16x2(fmaxf(__uint_as_float(w[0]), 0.f), fmaxf(__uint_as_float(w[1]), 0.f)),
-                                       pack_bf16x2(fmaxf(__uint_as_float(w[2]), 0.f), fmaxf(__uint_as_float(w[3]), 0.f)),
-                                       pack_bf16x2(fmaxf(__uint_as_float(w[4]), 0.f), fmaxf(__uint_as_float(w[5]), 0.f)),
-                                       pack_bf16x2(fmaxf(__uint_as_float(w[6]), 0.f), fmaxf(__uint_as_float(w[7]), 0.f)));
-            *reinterpret_cast<uint4*>(xy + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+            for (int q = 0; q < 4; ++q) {
+              float4 l4 = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (last >= 0) l4 = *reinterpret_cast<const float4*>(tl + c16 * 16 + 4 * q);
+              y[4 * q] = fmaxf(__uint_as_float(v[4 * q]) + l4.x, 0.f);
+              y[4 * q + 1] = fmaxf(__uint_as_float(v[4 * q + 1]) + l4.y, 0.f);
+              y[4 * q + 2] = fmaxf(__uint_as_float(v[4 * q + 2]) + l4.z, 0.f);
+              y[4 * q + 3] = fmaxf(__uint_as_float(v[4 * q + 3]) + l4.w, 0.f);
+            }
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+              const uint4 o = make_uint4(pack_bf16x2(y[8 * cc], y[8 * cc + 1]), pack_bf16x2(y[8 * cc + 2], y[8 * cc + 3]),
+                                         pack_bf16x2(y[8 * cc + 4], y[8 * cc + 5]), pack_bf16x2(y[8 * cc + 6], y[8 * cc + 7]));
+              *reinterpret_cast<uint4*>(xy + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+            }
           }
         }
         fence_proxy_async_smem();
@@ -659,11 +683,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             c_steps += 1;
             c_explore += pick >= 0 ? 1u : 0u;
             if (mask == 0) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
-            if (act != la) {  // move the last-action one-hot
-              if (la >= 0) *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
-              *reinterpret_cast<uint16_t*>(oh_col(3 + n + act)) = 0x3F80;
-              la = act;
-            }
+            la = act;
+            la_s[row] = act;  // read by both threads of the row in the next step's epilogue 1
             float* qrow = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
             if ((A & 1) == 0) {  // rows of an even number of floats start on 8-byte boundaries
 #pragma unroll
@@ -720,10 +741,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
           for (int cc = 0; cc < 4; ++cc)
             *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = make_uint4(0, 0, 0, 0);
-          if (half == 0 && la >= 0) {
-            *reinterpret_cast<uint16_t*>(oh_col(3 + n + la)) = 0;
-            la = -1;
-          }
+          if (half == 0) la = -1;
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
