@@ -256,6 +256,11 @@ void marl_actor_destroy(marl_actor_t* a);
  * mechanism works.  The CUDA context stays usable afterwards. */
 int marl_selftest_bounded_wait(void* stream, uint32_t poll_limit, uint32_t* status_out);
 
+/* Measurement helper (no counterpart in the paper): runs a dependency-free fp32 FMA loop on every SM and reports
+ * the best of three timed repetitions in TFLOP/s - the arithmetic bound of the fp32 actor path on this device
+ * at the clocks it actually sustains.  SYNCHRONISES the stream; takes a few tens of milliseconds. */
+int marl_measure_ffma_tflops(void* stream, double* tflops_out);
+
 /* Name of the step kernel in use: "ffma" or "tcgen05". */
 const char* marl_actor_kernel_name(const marl_actor_t* a);
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "marl_actor_set_trace", "marl_ring_view", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
     "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc", "marl_selftest_bounded_wait",
+    "marl_measure_ffma_tflops",
 ]
 
 
@@ -103,6 +104,7 @@ def load_library():
         lib.marl_rollout_staged.argtypes = [P, P, P, P, P, C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout_noalloc.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
+        lib.marl_measure_ffma_tflops.argtypes = [P, C.POINTER(C.c_double)]
         lib.marl_selftest_bounded_wait.argtypes = [P, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.marl_actor_set_trace.argtypes = [P, P, P, C.c_int32]
         lib.marl_ring_view.argtypes = [P, C.POINTER(RingView)]
@@ -140,6 +142,14 @@ def marl_actor_query_sizes(cfg: dict) -> dict:
     c = make_config(cfg)
     _check(load_library().marl_actor_query_sizes(C.byref(c), C.byref(s)))
     return {k: getattr(s, k) for k, _ in Sizes._fields_}
+
+
+def marl_measure_ffma_tflops() -> float:
+    """fp32 FMA peak of the current device under load, in TFLOP/s (measured by the library)."""
+    out = C.c_double(0)
+    stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().marl_measure_ffma_tflops(C.c_void_p(stream), C.byref(out)))
+    return float(out.value)
 
 
 def marl_selftest_bounded_wait(poll_limit: int = 20000) -> int:

@@ -23,11 +23,17 @@ constexpr int FF_THREADS = 256;
 constexpr int FF_QSTRIDE = 33;   // row stride of the Q tile (odd: one row per thread without conflicts)
 
 struct FfmaSmem {
-  int Dp, Hp;
-  size_t off_xs, off_ys, off_hs, off_hq, off_qs, off_mask, off_la, off_env, total;
+  int Dp, Hp, wsmem;
+  size_t off_xs, off_ys, off_hs, off_qs, off_mask, off_la, off_env, off_w, w_floats, total;
 };
 
-__host__ __device__ inline FfmaSmem ffma_smem_layout(int D, int H, int prec) {
+// Floats of the weight image kept in shared memory when it fits (hidden size 64): the k-major matrices
+// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2 [A][H], in this order.
+__host__ __device__ inline size_t ffma_weight_floats(int n, int D, int A, int H) {
+  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)A * H;
+}
+
+__host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H) {
   FfmaSmem s;
   int Dp = (D + 3) & ~3;
   if ((Dp & 31) == 0) Dp += 4;
@@ -37,12 +43,14 @@ __host__ __device__ inline FfmaSmem ffma_smem_layout(int D, int H, int prec) {
   s.off_xs = o; o += sizeof(float) * FF_RMAX * s.Dp;
   s.off_ys = o; o += sizeof(float) * FF_RMAX * s.Hp;
   s.off_hs = o; o += sizeof(float) * 2 * FF_RMAX * s.Hp;
-  s.off_hq = s.off_hs;  // fp32 precision: the operand copy is the state itself
-  if (prec == MARL_PRECISION_BF16) { s.off_hq = o; o += sizeof(float) * 2 * FF_RMAX * s.Hp; }
   s.off_qs = o; o += sizeof(float) * FF_RMAX * FF_QSTRIDE;
   s.off_mask = o; o += sizeof(uint32_t) * FF_RMAX;
   s.off_la = o; o += sizeof(int32_t) * FF_RMAX;
   s.off_env = o; o += 32 * FF_RMAX;  // per-environment scratch: see EnvSlot
+  s.off_w = o;
+  s.w_floats = ffma_weight_floats(n, D, A, H);
+  s.wsmem = (o + sizeof(float) * s.w_floats <= 227 * 1024) ? 1 : 0;  // resident weights if they fit
+  if (s.wsmem) o += sizeof(float) * s.w_floats;
   s.total = o;
   return s;
 }
@@ -58,13 +66,24 @@ struct EnvSlot {            // 32 bytes per environment of the tile
 
 __device__ __forceinline__ float sigmoid_accurate(float x) { return 1.0f / (1.0f + expf(-x)); }
 
+// Weight loads: from the shared-memory copy (WS) or through the read-only global path.
+template <bool WS>
+__device__ __forceinline__ float4 wload4(const float* ptr) {
+  if (WS) return *reinterpret_cast<const float4*>(ptr);
+  return __ldg(reinterpret_cast<const float4*>(ptr));
+}
+__device__ __forceinline__ float4 round4(float4 v, bool lowp) {
+  if (lowp) { v.x = bf16_round(v.x); v.y = bf16_round(v.y); v.z = bf16_round(v.z); v.w = bf16_round(v.w); }
+  return v;
+}
+
+template <bool WS>
 __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_constant__ ActorParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
-  const FfmaSmem sl = ffma_smem_layout(p.D, p.H, p.prec);
+  const FfmaSmem sl = ffma_smem_layout(p.n, p.D, p.A, p.H);
   float* xs = reinterpret_cast<float*>(smem + sl.off_xs);
   float* ys = reinterpret_cast<float*>(smem + sl.off_ys);
   float* hs = reinterpret_cast<float*>(smem + sl.off_hs);
-  float* hq = reinterpret_cast<float*>(smem + sl.off_hq);  // == hs in fp32 precision
   float* qs = reinterpret_cast<float*>(smem + sl.off_qs);
   uint32_t* masks = reinterpret_cast<uint32_t*>(smem + sl.off_mask);
   int32_t* la = reinterpret_cast<int32_t*>(smem + sl.off_la);
@@ -79,7 +98,17 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
   uint32_t st_bits = 0;
 
-  for (int i = tid; i < (int)(sl.total / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;
+  for (int i = tid; i < (int)(sl.off_w / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;
+  // weight pointers: the resident copy, or the k-major global arrays
+  const float *W1T = p.W1T, *WihT = p.WihT, *WhhT = p.WhhT, *W2 = p.W2;
+  if (WS) {
+    float* wsm = reinterpret_cast<float*>(smem + sl.off_w);
+    const size_t n1 = (size_t)(p.I + 4) * H, n2 = (size_t)H * H3, n3 = (size_t)A * H;
+    for (size_t i = tid; i < n1; i += FF_THREADS) wsm[i] = p.W1T[i];
+    for (size_t i = tid; i < n2; i += FF_THREADS) { wsm[n1 + i] = p.WihT[i]; wsm[n1 + n2 + i] = p.WhhT[i]; }
+    for (size_t i = tid; i < n3; i += FF_THREADS) wsm[n1 + 2 * n2 + i] = p.W2[i];
+    W1T = wsm; WihT = wsm + n1; WhhT = wsm + n1 + n2; W2 = wsm + n1 + 2 * n2;
+  }
   __syncthreads();
 
   for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
@@ -93,7 +122,6 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       const int r = idx / H, j = idx - r * H;
       const float v = p.h[(size_t)e0 * n * H + idx];
       hs[r * Hp + j] = v;
-      if (lowp) hq[r * Hp + j] = bf16_round(v);
     }
     for (int r = tid; r < FF_RMAX; r += FF_THREADS) la[r] = (r < R) ? p.last_action[e0 * n + r] : -1;
     if (tid < ne) {
@@ -175,7 +203,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xs + (ty + 16 * m) * Dp + k);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            const float4 w = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(k + kk) * H + j0));
+            const float4 w = wload4<WS>(W1T + (size_t)(k + kk) * H + j0);
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
               const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
@@ -190,11 +218,11 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         for (int m = 0; m < 4; ++m) {
           const int r = ty + 16 * m;
           const int ai = r % n;
-          const float4 wid = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(D + ai) * H + j0));
+          const float4 wid = wload4<WS>(W1T + (size_t)(D + ai) * H + j0);
           float4 o = make_float4(acc[m][0] + wid.x, acc[m][1] + wid.y, acc[m][2] + wid.z, acc[m][3] + wid.w);
           const int last = la[r];
           if (last >= 0) {
-            const float4 wl = __ldg(reinterpret_cast<const float4*>(p.W1T + (size_t)(D + n + last) * H + j0));
+            const float4 wl = wload4<WS>(W1T + (size_t)(D + n + last) * H + j0);
             o.x += wl.x; o.y += wl.y; o.z += wl.z; o.w += wl.w;
           }
           o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
@@ -225,18 +253,19 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         }
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
-          const float* act = pass == 0 ? ys : (hq + cur * hbuf);
-          const float* WT = pass == 0 ? p.WihT : p.WhhT;
+          const float* act = pass == 0 ? ys : (hs + cur * hbuf);
+          const float* WT = pass == 0 ? WihT : WhhT;
+          const bool rnd = lowp && pass == 1;  // the hidden state is stored in fp32; its operand copy is rounded here
           for (int k = 0; k < H; k += 4) {
             float4 v[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) v[m] = *reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k);
+            for (int m = 0; m < 4; ++m) v[m] = round4(*reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k), rnd);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
               const float* wrow = WT + (size_t)(k + kk) * H3 + j0;
-              const float4 wr = __ldg(reinterpret_cast<const float4*>(wrow));
-              const float4 wz = __ldg(reinterpret_cast<const float4*>(wrow + H));
-              const float4 wn = __ldg(reinterpret_cast<const float4*>(wrow + 2 * H));
+              const float4 wr = wload4<WS>(wrow);
+              const float4 wz = wload4<WS>(wrow + H);
+              const float4 wn = wload4<WS>(wrow + 2 * H);
 #pragma unroll
               for (int m = 0; m < 4; ++m) {
                 const float a = kk == 0 ? v[m].x : kk == 1 ? v[m].y : kk == 2 ? v[m].z : v[m].w;
@@ -269,9 +298,6 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             o[c] = fmaf(zg, hpv[c] - cand, cand);  // (1 - z) * cand + z * h
           }
           *reinterpret_cast<float4*>(hs + nxt * hbuf + r * Hp + j0) = make_float4(o[0], o[1], o[2], o[3]);
-          if (lowp)
-            *reinterpret_cast<float4*>(hq + nxt * hbuf + r * Hp + j0) =
-                make_float4(bf16_round(o[0]), bf16_round(o[1]), bf16_round(o[2]), bf16_round(o[3]));
         }
       }
       __syncthreads();
@@ -285,14 +311,14 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           const int a = part + 4 * m;
           acc[m] = a < A ? __ldg(p.b2 + a) : 0.f;
         }
-        const float* hv = hq + nxt * hbuf + r * Hp;
+        const float* hv = hs + nxt * hbuf + r * Hp;
         for (int k = 0; k < H; k += 4) {
-          const float4 v = *reinterpret_cast<const float4*>(hv + k);
+          const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
 #pragma unroll
           for (int m = 0; m < 8; ++m) {
             const int a = part + 4 * m;
             if (a < A) {
-              const float4 w = __ldg(reinterpret_cast<const float4*>(p.W2 + (size_t)a * H + k));
+              const float4 w = wload4<WS>(W2 + (size_t)a * H + k);
               acc[m] = fmaf(v.x, w.x, acc[m]);
               acc[m] = fmaf(v.y, w.y, acc[m]);
               acc[m] = fmaf(v.z, w.z, acc[m]);
@@ -365,7 +391,6 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         const int r = idx / H, j = idx - r * H;
         if (envs[r / n].reset) {
           hs[nxt * hbuf + r * Hp + j] = 0.f;
-          if (lowp) hq[nxt * hbuf + r * Hp + j] = 0.f;
         }
       }
       if (tid < R && envs[tid / n].reset) la[tid] = -1;
@@ -410,21 +435,22 @@ void ffma_tiling(int E, int n, int sms, int* ept, int* num_tiles) {
   *num_tiles = (E + per - 1) / per;
 }
 
-size_t ffma_smem_bytes(int D, int H, int prec) { return ffma_smem_layout(D, H, prec).total; }
+size_t ffma_smem_bytes(int n, int D, int A, int H) { return ffma_smem_layout(n, D, A, H).total; }
 
 // Returns the number of kernels launched or a negative cudaError.
 int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream) {
-  const size_t smem = ffma_smem_bytes(p.D, p.H, p.prec);
-  static size_t configured = 0;
-  if (smem > configured) {
-    const cudaError_t e =
-        cudaFuncSetAttribute(actor_ffma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const FfmaSmem sl = ffma_smem_layout(p.n, p.D, p.A, p.H);
+  auto kernel = sl.wsmem ? actor_ffma_kernel<true> : actor_ffma_kernel<false>;
+  static size_t configured[2] = {0, 0};
+  size_t& conf = configured[sl.wsmem];
+  if (sl.total > conf) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.total);
     if (e != cudaSuccess) return -(int)e;
-    configured = smem;
+    conf = sl.total;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;
-  actor_ffma_kernel<<<grid, FF_THREADS, smem, stream>>>(p);
+  kernel<<<grid, FF_THREADS, sl.total, stream>>>(p);
   const cudaError_t err = cudaGetLastError();
   return err == cudaSuccess ? 1 : -(int)err;
 }

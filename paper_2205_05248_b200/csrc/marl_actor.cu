@@ -16,7 +16,7 @@ namespace marl {
 int launch_env_generate(const marl_synth_env_t& env, int E, int n, int D, int A, uint32_t t0, int n_steps,
                         float* obs, uint8_t* avail, float* reward, uint8_t* done, int sms, cudaStream_t stream);
 void ffma_tiling(int E, int n, int sms, int* ept, int* num_tiles);
-size_t ffma_smem_bytes(int D, int H, int prec);
+size_t ffma_smem_bytes(int n, int D, int A, int H);
 int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream);
 // tensor-core kernel
 bool tc_supported(int n, int D, int A, int H, int prec);
