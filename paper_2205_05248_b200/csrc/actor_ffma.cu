@@ -21,6 +21,7 @@ namespace marl {
 constexpr int FF_RMAX = 64;      // rows per tile
 constexpr int FF_THREADS = 256;
 constexpr int FF_QSTRIDE = 33;   // row stride of the Q tile (odd: one row per thread without conflicts)
+constexpr int FF_PRE = 8;        // float4 registers per thread that hold the next step's observations
 
 struct FfmaSmem {
   int Dp, Hp, wsmem;
@@ -72,6 +73,12 @@ __device__ __forceinline__ float4 wload4(const float* ptr) {
   if (WS) return *reinterpret_cast<const float4*>(ptr);
   return __ldg(reinterpret_cast<const float4*>(ptr));
 }
+// Volatile, so that the request stays where it is written: a whole step before the value is used.
+__device__ __forceinline__ float4 ldg_nc_v4(const float4* ptr) {
+  float4 v;
+  asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr));
+  return v;
+}
 __device__ __forceinline__ float4 round4(float4 v, bool lowp) {
   if (lowp) { v.x = bf16_round(v.x); v.y = bf16_round(v.y); v.z = bf16_round(v.z); v.w = bf16_round(v.w); }
   return v;
@@ -111,11 +118,26 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   }
   __syncthreads();
 
+  // Observation tiles whose rows are whole float4s are requested one step ahead into registers, so that the
+  // global-memory latency is hidden behind the previous step's arithmetic.
+  const bool vec = (D % 4 == 0) && (reinterpret_cast<uintptr_t>(p.obs) % 16 == 0) && (FF_RMAX * D / 4 <= FF_THREADS * FF_PRE);
+  float4 pre[FF_PRE];
+
   for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
     const int e0 = tile * p.ept;
     const int ne = min(p.ept, p.E - e0);  // environments in this tile
     const int R = ne * n;                 // live rows
     int cur = 0;
+    auto prefetch_obs = [&](int s) {
+      const float4* src4 = reinterpret_cast<const float4*>(p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D);
+      const int nv = R * D / 4;
+#pragma unroll
+      for (int u = 0; u < FF_PRE; ++u) {
+        const int i4 = tid + u * FF_THREADS;
+        if (i4 < nv) pre[u] = ldg_nc_v4(src4 + i4);
+      }
+    };
+    if (vec) prefetch_obs(0);
 
     // ---- tile load: hidden state, last actions, ring cursors ----
     for (int idx = tid; idx < R * H; idx += FF_THREADS) {
@@ -147,7 +169,26 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       {
         const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
         const int nD = n * D;
-        for (int idx = tid; idx < R * D; idx += FF_THREADS) {
+        if (vec) {
+          const int nv = R * D / 4;
+#pragma unroll
+          for (int u = 0; u < FF_PRE; ++u) {
+            const int idx = (tid + u * FF_THREADS) * 4;
+            if (idx < nv * 4) {
+              asm volatile("" : "+f"(pre[u].x), "+f"(pre[u].y), "+f"(pre[u].z), "+f"(pre[u].w));  // first use is here
+              const int r = idx / D, d = idx - r * D;
+              const int el = idx / nD;
+              const float4 v = pre[u];
+              *reinterpret_cast<float4*>(xs + r * Dp + d) = round4(v, lowp);
+              const EnvSlot& es = envs[el];
+              if (es.ok)
+                *reinterpret_cast<float4*>(p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes +
+                                           p.rl.off_obs + (size_t)(idx - el * nD) * 4) = v;
+            }
+          }
+          if (s + 1 < p.T) prefetch_obs(s + 1);
+        }
+        for (int idx = tid; !vec && idx < R * D; idx += FF_THREADS) {
           const int r = idx / D, d = idx - r * D;
           const int el = idx / nD;
           const float v = src[idx];
