@@ -81,6 +81,49 @@ def test_config5_parity_small_E(H, prec, kernel):
     actor.destroy()
 
 
+def test_config5_full_size_bench_configuration():
+    """The workload and launch configuration that bench.py times (E=65536, H=64, bf16, T=64, 20 GB ring, tcgen05
+    kernel, one marl_rollout_staged call on pre-staged inputs); the oracle recomputes a seeded subset of
+    environments, and whole-batch properties are checked on everything."""
+    cfg = workloads.config(5)
+    w = workloads.make_weights(cfg)
+    actor = binding.Actor(cfg, kernel="auto", work_steps=1)
+    assert actor.kernel_name == "tcgen05"
+    actor.set_weights(w)
+    acts, q = actor.set_trace(cfg["T"])
+    staged = actor.env_generate(cfg["env"], 0, cfg["T"])
+    actor.rollout_staged(*staged, cfg["T"], cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+    torch.cuda.synchronize()
+    res = referee(cfg, w, actor, acts, q, env_ids=sample_envs(cfg["E"], 40, seed=5))
+    print(f"cfg5 full size: {res}")
+    status, counters = actor.status()
+    assert status == 0 and counters["agent_steps"] == cfg["E"] * cfg["n"] * cfg["T"]
+    # every chosen action is available, in every row of every step
+    avail = staged[1]
+    chosen = torch.gather(avail, 3, acts[: cfg["T"]].unsqueeze(-1).long()).squeeze(-1)
+    assert bool((chosen == 1).all())
+    # explore share ~ eps over 33.5 M rows
+    assert abs(counters["explored"] / counters["agent_steps"] - cfg["eps_start"]) < 1e-3
+    # slot headers against the done stream (one slot per environment here, so a new episode reuses the slot)
+    rv = actor.ring_view()
+    done = staged[3].long()                                            # [T][E]
+    T = cfg["T"]
+    idx = torch.arange(T, device=done.device)[:, None] * done          # step index where done, else 0
+    last_done = torch.where(done.any(0), idx.max(0).values, torch.full_like(idx[0], -1))
+    before = torch.where(idx < last_done[None, :], idx, torch.zeros_like(idx))   # done steps before the last one
+    prev_done = torch.where((done.sum(0) > 1), before.max(0).values, torch.full_like(last_done, -1))
+    closed_now = last_done == T - 1
+    want_len = torch.where(closed_now, last_done - prev_done, (T - 1) - last_done)
+    want_len = torch.where(want_len == 0, torch.ones_like(want_len), want_len)
+    got_len = rv["slot_len"].long()
+    open_or_closed = torch.where(closed_now, rv["slot_complete"].long() == 1, rv["slot_complete"].long() == 0)
+    assert bool(open_or_closed.all())
+    assert bool((got_len[~closed_now] == ((T - 1) - last_done)[~closed_now]).all())
+    assert bool((got_len[closed_now] == want_len[closed_now]).all())
+    del staged, acts, q
+    actor.destroy()
+
+
 def test_ragged_tiles_and_tiny_shapes():
     """Tile tails (E not a multiple of the tile), one agent, one action, one environment."""
     for over in (dict(E=37, n=5, C=74), dict(E=1, n=1, A=1, C=2), dict(E=150, n=7, A=32, D=3, C=150),
