@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--E", type=int, default=None)
     ap.add_argument("--H", type=int, default=None)
     ap.add_argument("--precision", default=None, choices=[None, "fp32", "bf16"])
-    ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor", "pipelined"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -298,7 +298,7 @@ def main():
     bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T) * E * n * T
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     flop_rate = flops_per_agent_step(cfg) * E * n * T / (kernel_ms * 1e-3) / 1e12
-    kname = "actor_%s_kernel" % ("tc" if actor.kernel_name == "tcgen05" else "ffma")
+    kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel"}.get(actor.kernel_name, "actor_ffma_kernel")
     if cfg["precision"] == "fp32":
         # the fp32 path is bound by plain FFMA arithmetic: peak measured on this device by the library's FMA loop
         ffma_peak = binding.marl_measure_ffma_tflops()

@@ -53,7 +53,11 @@ extern "C" {
 
 #define MARL_KERNEL_AUTO 0   /* tensor-core kernel where it is supported and the batch is large, else FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
-#define MARL_KERNEL_TENSOR 2 /* tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
+#define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
+#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, per-environment
+                                        * observation and availability blocks that are 16-byte multiples; create fails
+                                        * otherwise.  Inputs that are not 16-byte aligned fall back, per call, to
+                                        * the one-tile kernel where the shape allows it, else to the FFMA kernel */
 
 #define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
 #define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
@@ -261,7 +265,7 @@ int marl_selftest_bounded_wait(void* stream, uint32_t poll_limit, uint32_t* stat
  * at the clocks it actually sustains.  SYNCHRONISES the stream; takes a few tens of milliseconds. */
 int marl_measure_ffma_tflops(void* stream, double* tflops_out);
 
-/* Name of the step kernel in use: "ffma" or "tcgen05". */
+/* Name of the step kernel in use: "ffma", "tcgen05" (one-tile tensor-core kernel) or "tcgen05-pipelined". */
 const char* marl_actor_kernel_name(const marl_actor_t* a);
 
 /* Launches of library kernels enqueued by this actor since creation (all kernels, all entry points). */

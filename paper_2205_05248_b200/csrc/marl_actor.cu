@@ -26,6 +26,8 @@ void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b
                      void* dst_host);
 void tc_tiling(int E, int n, int sms, int* ept, int* num_tiles);
 int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream);
+bool tcp_supported(int n, int D, int A, int H, int prec);
+int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream);
 }  // namespace marl
 
 using namespace marl;
@@ -151,7 +153,7 @@ static int check_config(const marl_actor_config_t* c) {
     return fail(MARL_EINVAL, "ring_episodes must be a positive multiple of n_envs");
   if (c->precision != MARL_PRECISION_FP32 && c->precision != MARL_PRECISION_BF16)
     return fail(MARL_EINVAL, "unknown precision");
-  if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR) return fail(MARL_EINVAL, "unknown kernel");
+  if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR_PIPELINED) return fail(MARL_EINVAL, "unknown kernel");
   if (c->reserved != 0) return fail(MARL_EINVAL, "reserved must be 0");
   if ((double)c->n_envs * c->n_agents > 1.0e9) return fail(MARL_EINVAL, "n_envs * n_agents too large");
   return MARL_OK;
@@ -161,7 +163,8 @@ struct marl_actor {
   marl_actor_config_t cfg;
   cudaStream_t stream;
   int device, sms;
-  bool use_tc;
+  bool use_tc;   // a tensor-core kernel steps this actor
+  bool use_tcp;  // ... the pipelined one (falls back to the one-tile kernel for inputs it cannot bulk-copy)
   uint8_t *ring, *state, *work;
   bool own_ring, own_state, own_work;
   size_t work_bytes;
@@ -266,13 +269,16 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   a->launches = 0;
 
   const bool tc_ok = tc_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
-  if (cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) {
+  const bool tcp_ok = tcp_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
+  if ((cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) || (cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED && !tcp_ok)) {
     delete a;
     return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
   }
   // Below a couple of 128-row tiles the FFMA kernel, which spreads 64-row tiles over more SMs, is used.
-  a->use_tc = cfg->kernel == MARL_KERNEL_TENSOR ||
-              (cfg->kernel == MARL_KERNEL_AUTO && tc_ok && (long long)cfg->n_envs * cfg->n_agents >= 256);
+  const bool big = (long long)cfg->n_envs * cfg->n_agents >= 256;
+  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED;
+  a->use_tc = tc_ok && (cfg->kernel == MARL_KERNEL_TENSOR || cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED ||
+                        (cfg->kernel == MARL_KERNEL_AUTO && big));
 
   auto bind = [&](void* mem, size_t have, size_t need, uint8_t** dst, bool* own, const char* what) -> int {
     if (mem) {
@@ -360,7 +366,7 @@ int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, co
   memcpy(hp + a->wo.bhh, b_hh, sizeof(float) * 3 * H);
   memcpy(hp + a->wo.b2, b2, sizeof(float) * A);
   CU_TRY(cudaMemcpyAsync(a->state + a->so.wff, hp, a->wo.total, cudaMemcpyHostToDevice, a->stream));
-  if (tcb && tc_supported(n, D, A, H, a->cfg.precision)) {
+  if (tcb && (tc_supported(n, D, A, H, a->cfg.precision) || tcp_supported(n, D, A, H, a->cfg.precision))) {
     tc_pack_weights(n, D, A, H, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, hp + a->wo.total);
     CU_TRY(cudaMemcpyAsync(a->state + a->so.wpack, hp + a->wo.total, tcb, cudaMemcpyHostToDevice, a->stream));
   }
@@ -432,11 +438,13 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   p.avail_step_stride = (long long)c.n_envs * c.n_agents * c.n_actions;
   p.env_step_stride = c.n_envs;
   p.actions_out = actions_out;
-  int rc;
-  if (a->use_tc) {
+  int rc = 0;
+  if (a->use_tcp || a->use_tc) {
     tc_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
-    rc = launch_actor_tc(p, a->sms, a->stream);
-  } else {
+    if (a->use_tcp) rc = launch_actor_tcp(p, a->sms, a->stream);   // 0: these pointers cannot be bulk-copied
+    if (rc == 0 && a->use_tc) rc = launch_actor_tc(p, a->sms, a->stream);
+  }
+  if (rc == 0) {
     ffma_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
     rc = launch_actor_ffma(p, a->sms, a->stream);
   }
@@ -627,7 +635,10 @@ int marl_actor_reset(marl_actor_t* a) {
   return enqueue_reset(a);
 }
 
-const char* marl_actor_kernel_name(const marl_actor_t* a) { return (a && a->use_tc) ? "tcgen05" : "ffma"; }
+const char* marl_actor_kernel_name(const marl_actor_t* a) { 
+  if (!a) return "ffma";
+  return a->use_tcp ? "tcgen05-pipelined" : (a->use_tc ? "tcgen05" : "ffma");
+}
 
 uint64_t marl_actor_launch_count(const marl_actor_t* a) { return a ? a->launches : 0; }
 

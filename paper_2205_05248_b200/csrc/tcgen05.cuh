@@ -35,11 +35,26 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One wait attempt: the thread is suspended by the hardware until the phase completes or a time limit of the
+// order of `hint_ns` passes (no shared-memory polling traffic while it sleeps, immediate wake-up on completion).
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns = 20000u) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+
+// One non-blocking look at the barrier: true if the phase with this parity has completed.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
@@ -47,18 +62,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after `limit` polls (each poll may itself block for a hardware-defined time; the
-// default is about a second),
-// raises *abort_flag (shared) so that every later wait in the block returns at once, and reports failure.
+// Bounded wait: gives up after `limit` attempts (each may sleep up to the hint's 20 us, less if the hardware caps
+// it; the default bound is of the order of a second), raises *abort_flag (shared) so that every later wait in
+// the block returns at once, and reports failure.
 // The flag keeps the first failure's code: the barrier's byte offset in shared memory (low 20 bits) and the
 // waiting warp (bits 20..27), for diagnosis.  A kernel that saw a failure finishes its loops on garbage values
 // but keeps every index in range.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t limit = 300000u) {
+                                          uint32_t limit = 50000u) {
+#pragma unroll 1
   for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (i > 64) __nanosleep(32);
+    if (i > 4096) __nanosleep(64);  // a hardware that ignores the hint must not turn the wait into a hot spin
   }
   atomicCAS(const_cast<uint32_t*>(abort_flag), 0u, (smem_u32(bar) & 0xFFFFFu) | ((threadIdx.x >> 5) << 20) | 0x80000000u);
   return false;

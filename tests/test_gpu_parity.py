@@ -69,8 +69,8 @@ def test_configs_2_to_4_parity(k, n_ids):
     actor.destroy()
 
 
-@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "tensor"), (64, "bf16", "ffma"), (128, "bf16", "ffma"),
-                                           (64, "fp32", "ffma"), (128, "fp32", "ffma")])
+@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "pipelined"), (64, "bf16", "tensor"), (64, "bf16", "ffma"),
+                                           (128, "bf16", "ffma"), (64, "fp32", "ffma"), (128, "fp32", "ffma")])
 def test_config5_parity_small_E(H, prec, kernel):
     cfg = workloads.config(5, E=4096, H=H, precision=prec)
     cfg["T"] = 24
@@ -88,7 +88,7 @@ def test_config5_full_size_bench_configuration():
     cfg = workloads.config(5)
     w = workloads.make_weights(cfg)
     actor = binding.Actor(cfg, kernel="auto", work_steps=1)
-    assert actor.kernel_name == "tcgen05"
+    assert actor.kernel_name.startswith("tcgen05")
     actor.set_weights(w)
     acts, q = actor.set_trace(cfg["T"])
     staged = actor.env_generate(cfg["env"], 0, cfg["T"])
@@ -147,10 +147,66 @@ def test_tensor_kernel_ragged_tiles_and_tiny_shapes():
         actor.destroy()
 
 
-@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
-def test_done_every_step_and_never(kernel, prec):
+def _assert_same_rollout(a, acts_a, q_a, b, acts_b, q_b, tag=""):
+    """Two kernels that run the same arithmetic (the Q accumulation starts from the bias in one and ends with it in
+    the other, so Q may differ in the last bits): identical decisions, records, headers and state."""
+    assert torch.equal(acts_a, acts_b), tag
+    assert torch.allclose(q_a, q_b, rtol=1e-4, atol=2e-6), tag
+    ra, rb = a.ring_view(), b.ring_view()
+    for k in ("obs", "avail", "action", "reward", "done", "slot_epid", "slot_len", "slot_complete"):
+        assert torch.equal(ra[k], rb[k]), (tag, k)
+    assert torch.allclose(ra["q"], rb["q"], rtol=1e-4, atol=2e-6), tag
+    sa, sb = a.get_state(), b.get_state()
+    for key in ("last_action", "slot", "pos", "ep_count"):
+        assert torch.equal(sa[key], sb[key]), (tag, key)
+    assert torch.allclose(sa["h"], sb["h"], rtol=1e-4, atol=2e-6), tag
+    assert a.status() == b.status(), tag
+
+
+def test_pipelined_tensor_kernel_ragged_tiles_and_shapes():
+    """The pipelined tcgen05 kernel on tile tails, partial staging chunks (environment counts that are not
+    multiples of four), one tile, fewer tiles than blocks and more, agent counts that do not divide 128,
+    32 actions, observation widths that need padding to the MMA's K step."""
+    for over in (dict(E=130, n=8, D=80, A=14, C=260), dict(E=1, n=4, A=4, D=8, C=2), dict(E=37, n=16, A=5, D=16, C=74),
+                 dict(E=150, n=7, A=32, D=24, C=150), dict(E=9, n=32, A=2, D=40, C=9), dict(E=2500, n=8, A=6, D=72, C=2500),
+                 dict(E=333, n=5, A=16, D=88, C=333)):
+        cfg = workloads.small_config(H=64, L=7, T=20, precision="bf16", **over)
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="pipelined")
+        assert actor.kernel_name == "tcgen05-pipelined"
+        # the one-tile kernel does the same arithmetic: same decisions, same records
+        try:
+            one, acts1, q1 = run_gpu_rollout(cfg, w, kernel="tensor")
+        except binding.MarlError:      # its two full record buffers do not fit shared memory for this shape
+            one = None
+            assert over["D"] == 88
+        if one is not None:
+            _assert_same_rollout(actor, acts, q, one, acts1, q1, tag=str(over))
+            one.destroy()
+        referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
+        actor.destroy()
+
+
+def test_pipelined_and_one_tile_kernels_write_the_same_ring():
+    """Both tensor-core kernels run the same arithmetic: identical actions, records, headers and state (Q and h to
+    the last bits)."""
+    cfg = workloads.config(2, E=600)
+    cfg["T"] = 40
+    w = workloads.make_weights(cfg)
+    a, acts_a, q_a = run_gpu_rollout(cfg, w, kernel="pipelined")
+    b, acts_b, q_b = run_gpu_rollout(cfg, w, kernel="tensor")
+    assert a.kernel_name == "tcgen05-pipelined" and b.kernel_name == "tcgen05"
+    _assert_same_rollout(a, acts_a, q_a, b, acts_b, q_b)
+    a.destroy()
+    b.destroy()
+
+
+@pytest.mark.parametrize("kernel,prec,shape", [("ffma", "fp32", {}), ("tensor", "bf16", {}),
+                                               ("pipelined", "bf16", dict(n=4, A=8))])
+def test_done_every_step_and_never(kernel, prec, shape):
     for thr, L in ((1 << 24, 4), (0, 5)):
-        cfg = workloads.small_config(H=64, D=8, E=40, C=80, L=L, T=17, precision=prec, env=dict(done_thresh24=thr))
+        cfg = workloads.small_config(H=64, D=8, E=40, C=80, L=L, T=17, precision=prec, env=dict(done_thresh24=thr),
+                                     **shape)
         w = workloads.make_weights(cfg)
         actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
         res = referee(cfg, w, actor, acts, q, near_tie_budget=2e-3)
@@ -162,12 +218,13 @@ def test_done_every_step_and_never(kernel, prec):
         actor.destroy()
 
 
-@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
-def test_annealed_epsilon_and_split_rollouts_resume(kernel, prec):
+@pytest.mark.parametrize("kernel,prec,shape", [("ffma", "fp32", {}), ("tensor", "bf16", {}),
+                                               ("pipelined", "bf16", dict(n=8, A=6))])
+def test_annealed_epsilon_and_split_rollouts_resume(kernel, prec, shape):
     """eps schedule follows the global step; rollout(T) == rollout(a) + rollout(b); a checkpoint restored
     into a fresh handle continues identically."""
     cfg = workloads.small_config(H=64, D=16, E=64, C=128, L=9, T=30, eps_start=1.0, eps_end=0.05, anneal_steps=29,
-                                 precision=prec)
+                                 precision=prec, **shape)
     w = workloads.make_weights(cfg)
     one, a1, q1 = run_gpu_rollout(cfg, w, kernel=kernel)
     referee(cfg, w, one, a1, q1, near_tie_budget=2e-3)
@@ -195,13 +252,14 @@ def test_annealed_epsilon_and_split_rollouts_resume(kernel, prec):
         a.destroy()
 
 
-@pytest.mark.parametrize("kernel,prec", [("ffma", "fp32"), ("tensor", "bf16")])
-def test_step_api_equals_rollout_and_host_variant(kernel, prec):
+@pytest.mark.parametrize("kernel,prec,A", [("ffma", "fp32", 5), ("tensor", "bf16", 5), ("pipelined", "bf16", 12)])
+def test_step_api_equals_rollout_and_host_variant(kernel, prec, A):
     """T calls of marl_actor_step (device inputs) and of marl_actor_step_host (host inputs) reproduce
     marl_rollout: same actions, same ring, same state."""
-    cfg = workloads.small_config(H=64, D=24, E=50, n=4, C=100, L=8, T=12, precision=prec)
+    cfg = workloads.small_config(H=64, D=24, E=50, n=4, A=A, C=100, L=8, T=12, precision=prec)
     w = workloads.make_weights(cfg)
     ref, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
+    assert ref.kernel_name == {"ffma": "ffma", "tensor": "tcgen05", "pipelined": "tcgen05-pipelined"}[kernel]
     obs, avail, rew, done = ref.env_generate(cfg["env"], 0, cfg["T"])
     dev = binding.Actor(cfg, kernel=kernel)
     dev.set_weights(w)
@@ -296,8 +354,9 @@ def test_bounded_wait_gives_up_and_context_survives():
     assert st & binding.STATUS_TIMEOUT and st & 0x100
     x = torch.arange(8, device="cuda").sum().item()      # the context still works
     assert x == 28
-    cfg = workloads.small_config(H=64, D=8, precision="bf16", E=40, C=40)
-    w = workloads.make_weights(cfg)
-    actor, acts, q = run_gpu_rollout(cfg, w, kernel="tensor")
-    assert actor.status()[0] == 0                        # and a real rollout afterwards is clean
-    actor.destroy()
+    for kernel, shape in (("tensor", {}), ("pipelined", dict(n=4, A=8))):
+        cfg = workloads.small_config(H=64, D=8, precision="bf16", E=40, C=40, **shape)
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
+        assert actor.status()[0] == 0                    # and a real rollout afterwards is clean
+        actor.destroy()
