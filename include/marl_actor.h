@@ -51,7 +51,8 @@ extern "C" {
 #define MARL_PRECISION_FP32 0 /* fp32 weights, fp32 FFMA arithmetic */
 #define MARL_PRECISION_BF16 1 /* weight matrices and matmul operands rounded to bf16 (RNE), fp32 accumulate */
 
-#define MARL_KERNEL_AUTO 0   /* tensor-core kernel where it is supported and the batch is large, else FFMA */
+#define MARL_KERNEL_AUTO 0   /* a tensor-core kernel (the pipelined one where the shape allows it) where supported and
+                              * the batch is large, else FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
 #define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, per-environment

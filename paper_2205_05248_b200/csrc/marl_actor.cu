@@ -276,7 +276,7 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   }
   // Below a couple of 128-row tiles the FFMA kernel, which spreads 64-row tiles over more SMs, is used.
   const bool big = (long long)cfg->n_envs * cfg->n_agents >= 256;
-  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED;
+  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED || (cfg->kernel == MARL_KERNEL_AUTO && big && tcp_ok);
   a->use_tc = tc_ok && (cfg->kernel == MARL_KERNEL_TENSOR || cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED ||
                         (cfg->kernel == MARL_KERNEL_AUTO && big));
 
