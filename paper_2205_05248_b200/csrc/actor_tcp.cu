@@ -35,10 +35,27 @@
 
 namespace marl {
 
+// Phase timeline for tuning (compiled in only with -DMARL_TP_STAMPS): block 0 records the SM clock at its
+// hand-offs, per step, for a host-side reader.
+#ifdef MARL_TP_STAMPS
+__device__ unsigned long long g_tp_stamp[256 * 32];
+#define TP_STAMP(cond, step, id)                                                              \
+  do {                                                                                        \
+    if ((cond) && blockIdx.x == 0 && (step) < 256u) g_tp_stamp[(step) * 32 + (id)] = clock64(); \
+  } while (0)
+#else
+#define TP_STAMP(cond, step, id) \
+  do {                           \
+  } while (0)
+#endif
+
 constexpr int TP_THREADS = 512;
 constexpr int TP_CONV = 128;          // converter threads
 constexpr int TP_G = 4;               // environments per staging chunk
 constexpr int TP_MAX_STAGES = 8;
+// fc2 is four K = 16 steps.  Dependent tcgen05.mma on one accumulator run one after the other at a few hundred
+// cycles each whatever their width, so with 16 outputs the steps go to four accumulators (summed in epilogue 3).
+constexpr int TP_QPARTS = 4;
 constexpr int TP_DST_DEPTH = 16;      // steps of record addresses kept: the loads run at most TP_MAX_STAGES chunks (steps) ahead
 // Register split (setmaxnreg): launched with 128 registers per thread (512 * 128 = 65536); afterwards
 // 256 * 144 + 128 * 112 + 128 * 112 = 65536.
@@ -48,7 +65,7 @@ struct TpLayout {
   int32_t Dk, NQ, nchunk, ept, ohK, ohc, NS, pad_;
   uint32_t prefix_bytes, tail_bytes, chunk_bytes, obs_bytes, av_bytes;
   uint32_t off_W1, off_Wih, off_Whh, off_Bg, off_Bhn, off_W2, off_tab_la, wbytes;
-  uint32_t off_x, off_y, off_hb, off_oh, off_stage, off_tail, off_sel, off_la, off_close, off_closeany, off_rowenv, off_dstp, off_bar, total;
+  uint32_t off_x, off_y, off_hb, off_oh, off_stage, off_tail, off_sel, off_la, off_close, off_closeany, off_rowenv, off_dstp, off_tdst, off_bar, total;
 };
 
 struct TpBars {
@@ -86,6 +103,7 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.off_closeany = o; o += TP_DST_DEPTH * 4;
   L.off_rowenv = o; o += TC_ROWS * 4;
   L.off_dstp = o; o += TP_DST_DEPTH * 32 * 8;
+  L.off_tdst = o; o += 32 * 8;
   L.off_bar = o; o += (uint32_t)((sizeof(TpBars) + 15) & ~15u);
   L.off_stage = o;
   const uint32_t room = o + 32 < TC_SMEM_MAX ? TC_SMEM_MAX - o - 32 : 0;
@@ -106,6 +124,9 @@ bool tcp_supported(int n, int D, int A, int H, int prec) {
   // two tile-steps of chunks in flight at least, so that loads run well ahead of the network
   return L.NS >= 3 && L.total <= TC_SMEM_MAX;
 }
+
+// Tensor-memory columns of one Q buffer.
+__host__ __device__ constexpr uint32_t tp_qstride(int NQ) { return NQ == 16 ? TP_QPARTS * 16u : (uint32_t)NQ; }
 
 // One arrival per warp: every lane has made its writes (and proxy fences) before the warp-level barrier, lane 0
 // then arrives for all of them.  Arrivals on one mbarrier are serialised, so 8 instead of 256 matters.
@@ -181,6 +202,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
   int32_t* closeany_s = reinterpret_cast<int32_t*>(smem + L.off_closeany);  // [16] per step: some episode of the tile ends with it
   int32_t* rowenv_s = reinterpret_cast<int32_t*>(smem + L.off_rowenv);  // environment (within its chunk) of a chunk row
   unsigned long long* dstp_s = reinterpret_cast<unsigned long long*>(smem + L.off_dstp);  // [16][32] record address per step, environment
+  unsigned long long* tdst_s = reinterpret_cast<unsigned long long*>(smem + L.off_tdst);  // [32] tail addresses of the step being copied
   const float* tab_la = reinterpret_cast<const float*>(smem + L.off_tab_la);
   volatile uint32_t* abortf = &B->abort;
 
@@ -253,7 +275,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
       }
       for (int g = 0, s = 0; g < total; ++g) {
         const uint32_t par = (uint32_t)g & 1u;
-        const uint32_t qcol = TM_Q + par * NQ;  // Q accumulators alternate, so the next step's can be seeded early
+        const uint32_t qcol = TM_Q + par * tp_qstride(NQ);  // Q accumulators alternate, so the next step's can be seeded early
         if (!hside_issued) {
           // hidden operand in place: the tile prologue's, or the previous step's with closed episodes cleared
           if (s == 0) {
@@ -262,15 +284,18 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           } else {
             mbar_wait(&B->stepd, par ^ 1u, abortf);
           }
+          TP_STAMP(lane == 0, (uint32_t)g, 15);
           tp_issue_hside<NQ>(L, sb, tmem, lane, qcol);
         }
         mbar_wait(&B->yready, par, abortf);
+        TP_STAMP(lane == 0, (uint32_t)g, 8);
         tc_fence_after_sync();
         if (lane == 0) {
           const uint64_t d_y = smem_desc(sb + L.off_y, TC_LBO_A, 128), d_Wih = smem_desc(sb + L.off_Wih, TP_LBO_G, 128);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) mma_bf16(tmem + TM_R, d_y + ks * TP_K_A, d_Wih + ks * TP_K_G, idesc_bf16_f32(128, 192), 1);
           mma_commit(&B->grud);
+          TP_STAMP(true, (uint32_t)g, 9);
         }
         __syncwarp();
         // fc1 of the next step (possibly the next tile's first): its accumulator is free since epilogue 1 of
@@ -281,21 +306,27 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const uint32_t ready = __shfl_sync(0xFFFFFFFFu, lane == 0 ? (uint32_t)mbar_test_wait(&B->xready, par ^ 1u) : 0u, 0);
           if (ready) {
             tp_issue_fc1(L, sb, tmem, lane, &B->fc1d);
+            TP_STAMP(lane == 0, (uint32_t)g, 10);
             pending = false;
           }
         }
         mbar_wait(&B->hready, par, abortf);
+        TP_STAMP(lane == 0, (uint32_t)g, 11);
         tc_fence_after_sync();
         if (lane == 0) {
           const uint64_t d_h = smem_desc(sb + L.off_hb, TC_LBO_A, 128), d_W2 = smem_desc(sb + L.off_W2, NQ * 16, 128);
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) mma_bf16(tmem + qcol, d_h + ks * TP_K_A, d_W2 + ks * ((2 * NQ * 16) >> 4), idesc_bf16_f32(128, NQ), 1);
+          for (int ks = 0; ks < 4; ++ks)  // part 0 holds the bias already; parts 1..3 start from zero
+            mma_bf16(tmem + qcol + (NQ == 16 ? ks * NQ : 0), d_h + ks * TP_K_A, d_W2 + ks * ((2 * NQ * 16) >> 4), idesc_bf16_f32(128, NQ),
+                     (NQ == 16 && ks > 0) ? 0 : 1);
           mma_commit(&B->fc2d);
+          TP_STAMP(true, (uint32_t)g, 12);
         }
         __syncwarp();
         if (pending) {
           mbar_wait(&B->xready, par ^ 1u, abortf);
           tp_issue_fc1(L, sb, tmem, lane, &B->fc1d);
+          TP_STAMP(lane == 0, (uint32_t)g, 13);
         }
         // The next step's h-side products need only the new hidden state, which is in place unless an episode
         // of this tile ends with this step (its rows are cleared after fc2): issue them now, off the critical
@@ -306,7 +337,8 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         } else {
           // (published by the load warp before this step's inputs were requested: ordered before the fc1 operand)
           if (closeany_s[g & (TP_DST_DEPTH - 1)] == 0) {
-            tp_issue_hside<NQ>(L, sb, tmem, lane, TM_Q + (par ^ 1u) * NQ);
+            tp_issue_hside<NQ>(L, sb, tmem, lane, TM_Q + (par ^ 1u) * tp_qstride(NQ));
+            TP_STAMP(lane == 0, (uint32_t)g, 14);
             hside_issued = true;
           }
         }
@@ -400,6 +432,19 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           reward_next = p.reward[e];
           done_next = p.done[e];
         }
+        // Copies the tails of one step (buffer bb, record addresses in tdst_s) to the ring: 16 bytes per lane, the
+        // pieces of all environments in one flat loop.
+        auto copy_tails = [&](uint32_t bb) {
+          __syncwarp();
+          const uint32_t pieces = L.tail_bytes / 16u, total = (uint32_t)ne * pieces;
+          const uint32_t inv = 0xFFFFFFFFu / pieces + 1u;  // idx / pieces == umulhi(idx, inv) for idx < 2^16
+          for (uint32_t idx = lane; idx < total; idx += 32) {
+            const uint32_t env = __umulhi(idx, inv), pc = idx - env * pieces;
+            const unsigned long long d = tdst_s[env];
+            if (d) reinterpret_cast<uint4*>(d)[pc] = reinterpret_cast<const uint4*>(tails + bb * tail_set + env * L.tail_bytes)[pc];
+          }
+          __syncwarp();
+        };
         for (int s = 0; s < T; ++s) {
           const uint32_t b = it & 1;
           const float reward = reward_next;
@@ -419,21 +464,17 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             tl[t_done] = (uint8_t)done;
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive(&B->flags);
+          if (lane == 0) mbar_arrive(&B->flags);  // first: epilogue 3 of this step waits for it
+          TP_STAMP(lane == 0, it, 21);
+          if (s > 0) copy_tails(b ^ 1u);           // then the previous step's tails, off the critical path
           if (mine && s + 1 < T) {
             reward_next = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
             done_next = p.done[(size_t)(s + 1) * p.env_step_stride + e];
           }
           mbar_wait(&B->stepd, sd & 1, abortf);  // action and Q of step s are in the tail
+          TP_STAMP(lane == 0, it, 20);
           ++sd;
-          // the finished tails go to the ring, one environment at a time, 16 bytes per lane
-          for (int el = 0; el < ne; ++el) {
-            const unsigned long long d = __shfl_sync(0xFFFFFFFFu, dst, el);
-            if (d) {
-              const uint4* src = reinterpret_cast<const uint4*>(tails + b * tail_set + (uint32_t)el * L.tail_bytes);
-              for (uint32_t i = lane; i < L.tail_bytes / 16u; i += 32) reinterpret_cast<uint4*>(d)[i] = src[i];
-            }
-          }
+          tdst_s[lane] = dst;
           if (close) {
             p.slot_len[slot] = pos + 1;
             p.slot_complete[slot] = 1;
@@ -447,6 +488,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           }
           ++it;
         }
+        copy_tails((it - 1) & 1);  // the tile's last step
         if (mine && ok) {
           p.slot[e] = slot;
           p.pos[e] = pos;
@@ -511,6 +553,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         uint2* sel = sel_s + (it & 3) * TC_ROWS;
         // the operand buffer is free once fc1 of the previous step has finished reading it
         if (it > 0) mbar_wait(&B->fc1d, (it - 1) & 1, abortf);
+        TP_STAMP(ci == 0, it, 16);
         for (int c = cw; c < nck; c += TP_CONV / 32) {
           const int ge = min(TP_G, ne - c * TP_G);
           const int Rc = ge * n;         // rows of this chunk
@@ -577,6 +620,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         qbase += (uint32_t)nck;
         fence_proxy_async_smem();
         warp_arrive(&B->xready, lane);
+        TP_STAMP(ci == 0, it, 17);
         asm volatile("bar.sync 2, 128;" ::: "memory");  // the masks were written by the chunks' warps
         if (ci < ne * n) {
           const int rel = ci / n, rai = ci - rel * n;
@@ -586,6 +630,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           sel[ci].y = (uint32_t)pick;
         }
         warp_arrive(&B->selready[it & 3], lane);
+        TP_STAMP(ci == 0, it, 18);
         ++it;
       }
     }
@@ -642,6 +687,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         // ---- epilogue 1: y = relu(fc1 + W1[:, last action]) -> bf16 operand.  Bias and agent-id column are
         //      inside the GEMM; fc1 itself finished during the previous step. ----
         mbar_wait(&B->fc1d, par, abortf);
+        TP_STAMP(tid == 0, it, 0);
         tc_fence_after_sync();
         {
           // an episode that just ended has no last action
@@ -673,10 +719,12 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->yready, lane);
+        TP_STAMP(tid == 0, it, 1);
 
         // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand.
         //      The r and z accumulators hold half the pre-activation: sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 ----
         mbar_wait(&B->grud, par, abortf);
+        TP_STAMP(tid == 0, it, 2);
         tc_fence_after_sync();
 #pragma unroll
         for (int c16 = 0; c16 < 2; ++c16) {
@@ -706,20 +754,34 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->hready, lane);
+        TP_STAMP(tid == 0, it, 3);
 
         // ---- epilogue 3: the row owners choose and complete the record's tail ----
         mbar_wait(&B->flags, par, abortf);  // close flags of this step written, tail buffer free
+        TP_STAMP(tid == 0, it, 19);
         mbar_wait(&B->fc2d, par, abortf);   // (both halves: the hidden operand may be cleared below)
+        TP_STAMP(tid == 0, it, 4);
         tc_fence_after_sync();
         if (half == 0) {
           uint32_t qv[NQ];
-          const uint32_t qcol = TM_Q + par * NQ;
+          const uint32_t qcol = TM_Q + par * tp_qstride(NQ);
           tmem_ld16(tmem + lane_addr + qcol, *reinterpret_cast<uint32_t(*)[16]>(qv));
           if (NQ == 32) tmem_ld16(tmem + lane_addr + qcol + 16, *reinterpret_cast<uint32_t(*)[16]>(qv + NQ - 16));
+          if (NQ == 16) {  // the four K-step parts: (bias + part 0) + part 1 + part 2 + part 3
+            uint32_t q1[16], q2[16], q3[16];
+            tmem_ld16(tmem + lane_addr + qcol + 16, q1);
+            tmem_ld16(tmem + lane_addr + qcol + 32, q2);
+            tmem_ld16(tmem + lane_addr + qcol + 48, q3);
+            tmem_ld_wait();
+#pragma unroll
+            for (int a = 0; a < 16; ++a)
+              qv[a] = __float_as_uint((__uint_as_float(qv[a]) + __uint_as_float(q1[a])) + (__uint_as_float(q2[a]) + __uint_as_float(q3[a])));
+          }
           tmem_ld_wait();
           tc_fence_before_sync();
           if (is_row) {
             mbar_wait(&B->selready[it & 3], (it >> 2) & 1, abortf);
+            TP_STAMP(tid == 0, it, 5);
             const uint2 sp = sel_s[(it & 3) * TC_ROWS + row];
             const uint32_t mask = sp.x;
             const int pick = (int)sp.y;
@@ -773,6 +835,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           }
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
+        TP_STAMP(tid == 0, it, 6);
         // ---- a closed episode restarts from a zero hidden state and no last action ----
         if (live && close_s[b * 32 + el]) {
 #pragma unroll
@@ -785,6 +848,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->stepd, lane);
+        TP_STAMP(tid == 0, it, 7);
         ++it;
       }
 
@@ -834,3 +898,9 @@ int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream) {
 }
 
 }  // namespace marl
+
+#ifdef MARL_TP_STAMPS
+extern "C" int marl_tp_stamps(unsigned long long* out_host) {
+  return (int)cudaMemcpyFromSymbol(out_host, marl::g_tp_stamp, sizeof(unsigned long long) * 256 * 32);
+}
+#endif
