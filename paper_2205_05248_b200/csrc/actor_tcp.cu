@@ -14,11 +14,13 @@
 //     observations and its availability bytes are contiguous in the input arrays) issued up to NS chunks ahead
 //     of the network, across step and tile boundaries.  Bulk copies are kept few and large: their issue rate,
 //     not their bandwidth, limits a kernel that moves a few kilobytes per environment.
-//   * A warpgroup of converters takes each chunk out of staging once: the fp32 observations go to the ring
-//     (128-bit coalesced stores) and, rounded to bf16, into the fc1 operand; the availability bytes go to the
-//     ring and into the mask and Philox epsilon draw of every row.
-//   * fc1 of step s+1 needs only that operand, so it is issued during step s; per step the epilogue threads are
-//     left with: +last-action term, ReLU (epilogue 1) -> gate math (epilogue 2) -> masked arg-max (epilogue 3).
+//   * A warpgroup of converters (one warp per chunk, a step's chunks side by side) turns the fp32 observations
+//     into the bf16 fc1 operand, stores the availability bytes to the records and builds from them the mask and
+//     the Philox epsilon draw of every row; a store warp sends each environment's observations from staging to
+//     its record with one bulk store.
+//   * fc1 of step s+1 needs only that operand, and the h-side gate products of step s+1 only the new hidden
+//     state (unless an episode of the tile ends with step s), so both are issued during step s; per step the
+//     epilogue threads are left with: +last-action term, ReLU (epilogue 1) -> gate math (epilogue 2) -> masked arg-max (epilogue 3).
 //
 // Warp roles (512 threads): warps 0-7 epilogue (thread = one agent row x 32 hidden columns), warps 8-11
 // converters, warp 12 issues every tcgen05.mma, warp 13 issues the loads and runs the ring cursors ahead
