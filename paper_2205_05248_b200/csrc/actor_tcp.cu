@@ -728,29 +728,35 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         mbar_wait(&B->grud, par, abortf);
         TP_STAMP(tid == 0, it, 2);
         tc_fence_after_sync();
+        {
+          // Eight columns at a time; the accumulators of the next eight are requested before the gate math of the
+          // current ones (tcgen05.wait::ld waits for every load in flight, so the request follows the wait).
+          uint32_t g[2][4][8];  // [buffer][r, z, candidate-input, candidate-hidden][column]
+          auto request = [&](int c8, uint32_t (&d)[4][8]) {
+            const uint32_t col = (uint32_t)(cb + c8 * 8);
+            tmem_ld8(tmem + lane_addr + TM_R + col, d[0]);
+            tmem_ld8(tmem + lane_addr + TM_Z + col, d[1]);
+            tmem_ld8(tmem + lane_addr + TM_IN + col, d[2]);
+            tmem_ld8(tmem + lane_addr + TM_HN + col, d[3]);
+          };
+          request(0, g[0]);
 #pragma unroll
-        for (int c16 = 0; c16 < 2; ++c16) {
-          uint32_t vr[16], vz[16], vi[16], vh[16];
-          const uint32_t col = (uint32_t)(cb + c16 * 16);
-          tmem_ld16(tmem + lane_addr + TM_R + col, vr);
-          tmem_ld16(tmem + lane_addr + TM_Z + col, vz);
-          tmem_ld16(tmem + lane_addr + TM_IN + col, vi);
-          tmem_ld16(tmem + lane_addr + TM_HN + col, vh);
-          tmem_ld_wait();
+          for (int c8 = 0; c8 < 4; ++c8) {
+            tmem_ld_wait();
+            if (c8 + 1 < 4) request(c8 + 1, g[(c8 + 1) & 1]);
+            uint32_t(&v)[4][8] = g[c8 & 1];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float rg = fmaf(0.5f, tanh_fast(__uint_as_float(vr[j])), 0.5f);
-            const float zg = fmaf(0.5f, tanh_fast(__uint_as_float(vz[j])), 0.5f);
-            const float cand = tanh_fast(fmaf(rg, __uint_as_float(vh[j]), __uint_as_float(vi[j])));
-            const float hp = h[c16 * 16 + j];
-            h[c16 * 16 + j] = fmaf(zg, hp - cand, cand);  // (1 - z) * cand + z * h
-          }
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const float* hv = h + c16 * 16 + 8 * cc;
+            for (int j = 0; j < 8; ++j) {
+              const float rg = fmaf(0.5f, tanh_fast(__uint_as_float(v[0][j])), 0.5f);
+              const float zg = fmaf(0.5f, tanh_fast(__uint_as_float(v[1][j])), 0.5f);
+              const float cand = tanh_fast(fmaf(rg, __uint_as_float(v[3][j]), __uint_as_float(v[2][j])));
+              const float hp = h[c8 * 8 + j];
+              h[c8 * 8 + j] = fmaf(zg, hp - cand, cand);  // (1 - z) * cand + z * h
+            }
+            const float* hv = h + c8 * 8;
             const uint4 o = make_uint4(pack_bf16x2(hv[0], hv[1]), pack_bf16x2(hv[2], hv[3]), pack_bf16x2(hv[4], hv[5]),
                                        pack_bf16x2(hv[6], hv[7]));
-            *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + c16 * 2 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
+            *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + c8) * TC_LBO_A + (uint32_t)row * 16u) = o;
           }
         }
         fence_proxy_async_smem();
