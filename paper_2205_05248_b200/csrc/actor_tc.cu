@@ -40,7 +40,7 @@ bool tc_supported(int n, int D, int A, int H, int prec) {
 }
 
 size_t tc_wpack_bytes(int n, int D, int A, int H) {
-  if (H != TC_H || D % 8 != 0 || n < 1 || n > 32 || A < 1 || A > 32) return 0;
+  if (H != TC_H || D < 1 || D > 256 || n < 1 || n > 32 || A < 1 || A > 32) return 0;  // (a layout question only)
   return tc_layout(n, D, A, rec_bytes_of(n, D, A)).wbytes;
 }
 

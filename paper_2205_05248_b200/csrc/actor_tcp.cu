@@ -64,7 +64,7 @@ constexpr int TP_DST_DEPTH = 16;      // steps of record addresses kept: the loa
 constexpr int TP_REGS_EPI = 144, TP_REGS_CONV = 112, TP_REGS_SVC = 112;
 
 struct TpLayout {
-  int32_t Dk, NQ, nchunk, ept, ohK, ohc, NS, pad_;
+  int32_t Dk, NQ, nchunk, ept, ohK, ohc, NS, plain;
   uint32_t prefix_bytes, tail_bytes, chunk_bytes, obs_bytes, av_bytes;
   uint32_t off_W1, off_Wih, off_Whh, off_Bg, off_Bhn, off_W2, off_tab_la, wbytes;
   uint32_t off_x, off_y, off_hb, off_oh, off_stage, off_tail, off_sel, off_la, off_close, off_closeany, off_rowenv, off_dstp, off_tdst, off_bar, total;
@@ -90,8 +90,13 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.off_W2 = W.off_W2; L.off_tab_la = W.off_tab_la; L.wbytes = W.wbytes;
   L.obs_bytes = (uint32_t)(n * D) * 4u;
   L.av_bytes = (uint32_t)(n * A);
-  L.prefix_bytes = L.obs_bytes + L.av_bytes;
-  L.tail_bytes = (uint32_t)rec_bytes - L.prefix_bytes;
+  L.prefix_bytes = L.obs_bytes + L.av_bytes;  // of one environment in staging: [obs of the chunk | avail of the chunk]
+  // Shapes whose per-environment blocks are not 16-byte multiples ("plain"): whole chunks still are (4 n D floats,
+  // 4 n A bytes with n A a multiple of 4), so they load the same way, in tiles of whole chunks; the converters then
+  // read and store observations word by word instead of the store warp's bulk stores.
+  L.plain = (D % 8 != 0 || (n * A) % 16 != 0) ? 1 : 0;
+  if (L.plain) L.ept = L.ept / TP_G * TP_G;
+  L.tail_bytes = (uint32_t)rec_bytes - (up16(L.obs_bytes) + up16(L.av_bytes));
   L.chunk_bytes = TP_G * L.prefix_bytes;
   uint32_t o = L.wbytes;
   L.off_x = o; o += up16((uint32_t)L.nchunk * TC_LBO_X);
@@ -116,15 +121,15 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   return L;
 }
 
-// Shapes this kernel takes: those of the one-tile kernel whose per-environment observation and availability
-// blocks can be bulk-copied (16-byte multiples) and whose tiles have at most 32 environments (one lane each).
+// Shapes this kernel takes: at least 4 agents (tiles of at most 32 environments, one lane each) and chunks of
+// four environments whose observation and availability blocks are 16-byte multiples.
 bool tcp_supported(int n, int D, int A, int H, int prec) {
   if (prec != MARL_PRECISION_BF16 || H != TC_H) return false;
-  if (D % 8 != 0 || D > 256 || n < 4 || n > 32 || A < 1 || A > 32) return false;
-  if ((n * A) % 16 != 0) return false;
+  if (D < 1 || D > 256 || n < 4 || n > 32 || A < 1 || A > 32) return false;
+  if ((n * A) % 4 != 0) return false;  // a chunk's availability bytes must be a 16-byte multiple
   const TpLayout L = tp_layout(n, D, A, rec_bytes_of(n, D, A));
   // two tile-steps of chunks in flight at least, so that loads run well ahead of the network
-  return L.NS >= 3 && L.total <= TC_SMEM_MAX;
+  return L.ept >= TP_G && L.NS >= 3 && L.total <= TC_SMEM_MAX;
 }
 
 // Tensor-memory columns of one Q buffer.
@@ -515,7 +520,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             mbar_wait(&B->full[qslot], qpar, abortf);
             if (lane < ge) {
               const unsigned long long rec = dstp_s[(kstep & (TP_DST_DEPTH - 1)) * 32 + c * TP_G + lane];
-              if (rec) bulk_store(reinterpret_cast<void*>(rec), stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes, L.obs_bytes);
+              if (rec && !L.plain) bulk_store(reinterpret_cast<void*>(rec), stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes, L.obs_bytes);
             }
             bulk_commit();
             // every lane commits one (possibly empty) group per chunk, so "all but the latest" covers chunk q - 1
@@ -565,6 +570,25 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const unsigned long long* recs = dstp_s + (it & (TP_DST_DEPTH - 1)) * 32 + c * TP_G;  // this chunk's records
           mbar_wait(&B->full[qslot], qpar, abortf);
           const int items = Rc * L.nchunk;
+          if (L.plain) {
+            // rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record
+            for (int j = lane; j < items; j += 32) {
+              const int rr = (int)__umulhi((uint32_t)j, inv_nchunk), cc = j - rr * L.nchunk;
+              const int envc = rowenv_s[rr];
+              const unsigned long long rec = recs[envc];
+              const float* srow = reinterpret_cast<const float*>(src) + rr * D;
+              float* drow = reinterpret_cast<float*>(rec) + (rr - envc * n) * D;
+              float v[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int col = cc * 8 + k;
+                v[k] = col < D ? srow[col] : 0.f;
+                if (rec && col < D) drow[col] = v[k];
+              }
+              *reinterpret_cast<uint4*>(xb + (uint32_t)cc * TC_LBO_X + (uint32_t)(r0 + rr) * 16u) =
+                  make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+            }
+          } else
           for (int j = lane; j < items; j += 64) {
             float4 v[2][2];
             int rr[2], cc[2];
@@ -593,7 +617,14 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             }
           }
           const uint8_t* avs = src + TP_G * L.obs_bytes;  // the chunk's availability bytes, rows contiguous
-          {
+          if (L.plain) {
+            const uint32_t per_env = L.av_bytes / 4u;  // n A is a multiple of 4
+            for (uint32_t i = lane; i < (uint32_t)ge * per_env; i += 32) {
+              const uint32_t envc = i / per_env;
+              const unsigned long long rec = recs[envc];
+              if (rec) reinterpret_cast<uint32_t*>(rec + p.rl.off_avail)[i - envc * per_env] = reinterpret_cast<const uint32_t*>(avs)[i];
+            }
+          } else {
             const uint32_t per_env = L.av_bytes / 16u;
             for (uint32_t i = lane; i < (uint32_t)ge * per_env; i += 32) {
               const uint32_t envc = i / per_env;
@@ -886,10 +917,14 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 
 // Returns the number of kernels launched, 0 if this launch's pointers do not meet the kernel's alignment
 // needs (the caller then uses the one-tile kernel), or a negative cudaError.
-int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream) {
-  const TpLayout L = tp_layout(p.n, p.D, p.A, (int)p.rl.rec_bytes);
+int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
+  const TpLayout L = tp_layout(p_in.n, p_in.D, p_in.A, (int)p_in.rl.rec_bytes);
+  ActorParams p = p_in;
+  p.ept = L.ept;  // (tiles of whole chunks for the plain shapes)
+  p.num_tiles = (p.E + L.ept - 1) / L.ept;
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
+  if (L.plain && p.E % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
   auto kernel = L.NQ == 16 ? actor_tcp_kernel<16> : actor_tcp_kernel<32>;
   static uint32_t configured[2] = {0, 0};
   uint32_t& conf = configured[L.NQ == 16 ? 0 : 1];
