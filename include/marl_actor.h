@@ -55,10 +55,12 @@ extern "C" {
                               * the batch is large, else FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
-#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, per-environment
-                                        * observation and availability blocks that are 16-byte multiples; create fails
-                                        * otherwise.  Inputs that are not 16-byte aligned fall back, per call, to
-                                        * the one-tile kernel where the shape allows it, else to the FFMA kernel */
+#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, n_agents * n_actions
+                                        * a multiple of 4; create fails otherwise.  Inputs that are not 16-byte
+                                        * aligned (or, where an environment's observation or availability block is
+                                        * not a 16-byte multiple, an environment count that is not a multiple of 4)
+                                        * fall back, per call, to the one-tile kernel where the shape allows it,
+                                        * else to the FFMA kernel */
 
 #define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
 #define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
