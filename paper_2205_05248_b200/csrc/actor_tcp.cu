@@ -65,7 +65,7 @@ constexpr int TP_REGS_EPI = 144, TP_REGS_CONV = 112, TP_REGS_SVC = 112;
 
 struct TpLayout {
   int32_t Dk, NQ, nchunk, ept, ohK, ohc, NS, plain;
-  uint32_t prefix_bytes, tail_bytes, chunk_bytes, obs_bytes, av_bytes;
+  uint32_t prefix_bytes, tail_bytes, chunk_bytes, obs_bytes, av_bytes, rs_env, rs_bytes, off_rstage;
   uint32_t off_W1, off_Wih, off_Whh, off_Bg, off_Bhn, off_W2, off_tab_la, wbytes;
   uint32_t off_x, off_y, off_hb, off_oh, off_stage, off_tail, off_sel, off_la, off_close, off_closeany, off_rowenv, off_dstp, off_tdst, off_bar, total;
 };
@@ -113,11 +113,17 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.off_tdst = o; o += 32 * 8;
   L.off_bar = o; o += (uint32_t)((sizeof(TpBars) + 15) & ~15u);
   L.off_stage = o;
+  // plain shapes: the converters also lay the observations out as the records want them (each environment's block
+  // padded to 16 bytes), one image per staging slot, for the store warp's bulk stores
+  L.rs_env = L.plain ? up16(L.obs_bytes) : 0;
+  L.rs_bytes = TP_G * L.rs_env;
   const uint32_t room = o + 32 < TC_SMEM_MAX ? TC_SMEM_MAX - o - 32 : 0;
-  int ns = (int)(room / L.chunk_bytes);
+  int ns = (int)(room / (L.chunk_bytes + L.rs_bytes));
   if (ns > TP_MAX_STAGES) ns = TP_MAX_STAGES;
+  if (ns < 0) ns = 0;
   L.NS = ns;
-  L.total = o + (uint32_t)(ns > 0 ? ns : 0) * L.chunk_bytes + 32;  // (+32: the mask words read a few bytes past a row)
+  L.off_rstage = o + (uint32_t)ns * L.chunk_bytes + 32;  // (+32: the mask words read a few bytes past a row)
+  L.total = L.off_rstage + (uint32_t)ns * L.rs_bytes;
   return L;
 }
 
@@ -246,6 +252,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
   if (warp == 12) tmem_alloc(&B->tmem_base, TM_COLS);
   // operands, tails and hand-off arrays start as zeros (padding bytes of every stored record stay zero)
   for (uint32_t i = L.off_x / 16 + tid; i < L.off_bar / 16; i += TP_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  for (uint32_t i = L.off_rstage / 16 + tid; i < L.total / 16; i += TP_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   if (tid < TC_ROWS) {
     // one-hot operand tile: three ones (bias columns) and the agent's own column; the same for every tile
@@ -517,10 +524,13 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         for (int s = 0; s < T; ++s, ++kstep) {
           for (int c = 0; c < nck; ++c) {
             const int ge = min(TP_G, ne - c * TP_G);
-            mbar_wait(&B->full[qslot], qpar, abortf);
+            // plain shapes: the image the converters wrote, once they are done with the chunk; else the staged block
+            mbar_wait(L.plain ? &B->cfree[qslot] : &B->full[qslot], qpar, abortf);
             if (lane < ge) {
               const unsigned long long rec = dstp_s[(kstep & (TP_DST_DEPTH - 1)) * 32 + c * TP_G + lane];
-              if (rec && !L.plain) bulk_store(reinterpret_cast<void*>(rec), stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes, L.obs_bytes);
+              const uint8_t* from = L.plain ? smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)lane * L.rs_env
+                                            : stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes;
+              if (rec) bulk_store(reinterpret_cast<void*>(rec), from, L.plain ? L.rs_env : L.obs_bytes);
             }
             bulk_commit();
             // every lane commits one (possibly empty) group per chunk, so "all but the latest" covers chunk q - 1
@@ -571,19 +581,18 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           mbar_wait(&B->full[qslot], qpar, abortf);
           const int items = Rc * L.nchunk;
           if (L.plain) {
-            // rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record
+            // rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record image
             for (int j = lane; j < items; j += 32) {
               const int rr = (int)__umulhi((uint32_t)j, inv_nchunk), cc = j - rr * L.nchunk;
               const int envc = rowenv_s[rr];
-              const unsigned long long rec = recs[envc];
               const float* srow = reinterpret_cast<const float*>(src) + rr * D;
-              float* drow = reinterpret_cast<float*>(rec) + (rr - envc * n) * D;
+              float* drow = reinterpret_cast<float*>(smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)envc * L.rs_env) + (rr - envc * n) * D;
               float v[8];
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
                 const int col = cc * 8 + k;
                 v[k] = col < D ? srow[col] : 0.f;
-                if (rec && col < D) drow[col] = v[k];
+                if (col < D) drow[col] = v[k];
               }
               *reinterpret_cast<uint4*>(xb + (uint32_t)cc * TC_LBO_X + (uint32_t)(r0 + rr) * 16u) =
                   make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
@@ -647,6 +656,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             }
             sel[r0 + rc].x = (uint32_t)(bits >> (off & 3u)) & amask;
           }
+          if (L.plain) fence_proxy_async_smem();  // the record image is read by the store warp's bulk stores
           __syncwarp();
           if (lane == 0) mbar_arrive(&B->cfree[qslot]);
         }
