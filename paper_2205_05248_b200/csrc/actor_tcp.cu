@@ -113,9 +113,9 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.off_tdst = o; o += 32 * 8;
   L.off_bar = o; o += (uint32_t)((sizeof(TpBars) + 15) & ~15u);
   L.off_stage = o;
-  // plain shapes: the converters also lay the observations out as the records want them (each environment's block
-  // padded to 16 bytes), one image per staging slot, for the store warp's bulk stores
-  L.rs_env = L.plain ? up16(L.obs_bytes) : 0;
+  // plain shapes: the converters also lay observations and availability bytes out as the records want them (each
+  // block padded to 16 bytes), one image per staging slot, for the store warp's bulk stores
+  L.rs_env = L.plain ? up16(L.obs_bytes) + up16(L.av_bytes) : 0;  // the record's prefix [obs | avail], padded as in the ring
   L.rs_bytes = TP_G * L.rs_env;
   const uint32_t room = o + 32 < TC_SMEM_MAX ? TC_SMEM_MAX - o - 32 : 0;
   int ns = (int)(room / (L.chunk_bytes + L.rs_bytes));
@@ -628,10 +628,9 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const uint8_t* avs = src + TP_G * L.obs_bytes;  // the chunk's availability bytes, rows contiguous
           if (L.plain) {
             const uint32_t per_env = L.av_bytes / 4u;  // n A is a multiple of 4
-            for (uint32_t i = lane; i < (uint32_t)ge * per_env; i += 32) {
-              const uint32_t envc = i / per_env;
-              const unsigned long long rec = recs[envc];
-              if (rec) reinterpret_cast<uint32_t*>(rec + p.rl.off_avail)[i - envc * per_env] = reinterpret_cast<const uint32_t*>(avs)[i];
+            for (int envc = 0; envc < ge; ++envc) {
+              uint32_t* img = reinterpret_cast<uint32_t*>(smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)envc * L.rs_env + p.rl.off_avail);
+              for (uint32_t i = lane; i < per_env; i += 32) img[i] = reinterpret_cast<const uint32_t*>(avs)[(uint32_t)envc * per_env + i];
             }
           } else {
             const uint32_t per_env = L.av_bytes / 16u;
