@@ -442,7 +442,8 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   if (a->use_tcp || a->use_tc) {
     tc_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
     if (a->use_tcp) rc = launch_actor_tcp(p, a->sms, a->stream);   // 0: these pointers cannot be bulk-copied
-    if (rc == 0 && a->use_tc) rc = launch_actor_tc(p, a->sms, a->stream);
+    // (the one-tile kernel bulk-copies the observations too; it copes with unaligned availability bytes itself)
+    if (rc == 0 && a->use_tc && reinterpret_cast<uintptr_t>(obs) % 16 == 0) rc = launch_actor_tc(p, a->sms, a->stream);
   }
   if (rc == 0) {
     ffma_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);

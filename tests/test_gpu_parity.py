@@ -362,3 +362,44 @@ def test_bounded_wait_gives_up_and_context_survives():
         actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
         assert actor.status()[0] == 0                    # and a real rollout afterwards is clean
         actor.destroy()
+
+
+def test_pipelined_kernel_falls_back_on_unaligned_inputs():
+    """Inputs that are not 16-byte aligned cannot be bulk-copied: a step with unaligned availability bytes runs on
+    the one-tile kernel, one with unaligned observations on the FFMA kernel, each with that kernel's exact results;
+    the next aligned step is back on the pipelined kernel."""
+    cfg = workloads.small_config(H=64, D=24, E=40, n=4, A=12, C=80, L=8, T=3, precision="bf16")
+    w = workloads.make_weights(cfg)
+    pipe, tens, ffma = (binding.Actor(cfg, kernel=k) for k in ("pipelined", "tensor", "ffma"))
+    for a in (pipe, tens, ffma):
+        a.set_weights(w)
+    obs, avail, rew, done = pipe.env_generate(cfg["env"], 0, 3)
+
+    def shifted(t, elems):                      # a copy that starts `elems` elements into a fresh allocation
+        big = torch.empty(t.numel() + 64, dtype=t.dtype, device=t.device)
+        out = big[elems:elems + t.numel()].view(t.shape)
+        out.copy_(t)
+        return out
+
+    # step 0: unaligned availability bytes -> one-tile kernel
+    av = shifted(avail[0], 4)
+    assert av.data_ptr() % 16 != 0
+    a0 = pipe.step(obs[0], av, rew[0], done[0], cfg["eps_start"])
+    assert torch.equal(a0, tens.step(obs[0], avail[0], rew[0], done[0], cfg["eps_start"]))
+    ffma.step(obs[0], avail[0], rew[0], done[0], cfg["eps_start"])
+    # step 1: unaligned observations -> FFMA kernel (from the tensor-core kernels' state: compare decisions only where
+    # the hidden states agree to the tolerance, i.e. run the FFMA actor from the same state)
+    st = pipe.get_state()
+    ffma.set_state(st)
+    ffma.ring_mem.copy_(pipe.ring_mem)
+    ob = shifted(obs[1], 1)
+    assert ob.data_ptr() % 16 != 0
+    a1 = pipe.step(ob, avail[1], rew[1], done[1], cfg["eps_start"])
+    assert torch.equal(a1, ffma.step(obs[1], avail[1], rew[1], done[1], cfg["eps_start"]))
+    torch.cuda.synchronize()
+    assert torch.equal(pipe.ring_mem, ffma.ring_mem)
+    # step 2: aligned again
+    a2 = pipe.step(obs[2], avail[2], rew[2], done[2], cfg["eps_start"])
+    assert a2.shape == a1.shape and pipe.status()[0] == 0
+    for a in (pipe, tens, ffma):
+        a.destroy()
