@@ -296,11 +296,13 @@ def test_determinism_same_seed_same_bytes():
     b.destroy()
 
 
-def test_no_available_action_is_reported_not_fatal():
+@pytest.mark.parametrize("kernel,shape", [("ffma", dict(n=2)), ("tensor", dict(n=4, A=8, D=8, precision="bf16")),
+                                          ("pipelined", dict(n=4, A=8, D=8, precision="bf16"))])
+def test_no_available_action_is_reported_not_fatal(kernel, shape):
     """A row whose mask is all zero takes action 0, sets the status bit and counts it."""
-    cfg = workloads.small_config(H=64, E=6, n=2, C=6, L=8, T=1)
+    cfg = workloads.small_config(H=64, E=6, C=6, L=8, T=1, **shape)
     w = workloads.make_weights(cfg)
-    actor = binding.Actor(cfg, kernel="ffma")
+    actor = binding.Actor(cfg, kernel=kernel)
     actor.set_weights(w)
     obs, avail, rew, done = actor.env_generate(cfg["env"], 0, 1)
     avail[0, 3, 1, :] = 0
@@ -310,15 +312,19 @@ def test_no_available_action_is_reported_not_fatal():
     assert int(acts[3, 1]) == 0
     sess = oracle.Session(cfg, w, np.arange(cfg["E"]))
     o_acts, _ = sess.step(obs[0].cpu().numpy(), avail[0].cpu().numpy(), rew[0].cpu().numpy(), done[0].cpu().numpy(), 0.0)
-    assert np.array_equal(acts.cpu().numpy(), o_acts) and sess.counters[oracle.CNT_NO_AVAIL] == 1
+    assert sess.counters[oracle.CNT_NO_AVAIL] == 1 and int(o_acts[3, 1]) == 0
+    if kernel == "ffma":                     # (the bf16 kernels may differ from the oracle in a near-tie elsewhere)
+        assert np.array_equal(acts.cpu().numpy(), o_acts)
     actor.destroy()
 
 
-def test_bad_cursor_sets_status_and_skips():
+@pytest.mark.parametrize("kernel,shape", [("ffma", {}), ("tensor", dict(n=4, A=8, D=8, precision="bf16")),
+                                          ("pipelined", dict(n=4, A=8, D=8, precision="bf16"))])
+def test_bad_cursor_sets_status_and_skips(kernel, shape):
     """A corrupted ring cursor handed in through set_state is detected; nothing is written out of range."""
-    cfg = workloads.small_config(H=64, E=4, C=4, L=8, T=2)
+    cfg = workloads.small_config(H=64, E=4, C=4, L=8, T=2, **shape)
     w = workloads.make_weights(cfg)
-    actor = binding.Actor(cfg, kernel="ffma")
+    actor = binding.Actor(cfg, kernel=kernel)
     actor.set_weights(w)
     st = actor.get_state()
     bad = {k: (v.clone() if torch.is_tensor(v) else v) for k, v in st.items()}
