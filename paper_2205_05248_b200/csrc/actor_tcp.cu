@@ -628,9 +628,11 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const uint8_t* avs = src + TP_G * L.obs_bytes;  // the chunk's availability bytes, rows contiguous
           if (L.plain) {
             const uint32_t per_env = L.av_bytes / 4u;  // n A is a multiple of 4
-            for (int envc = 0; envc < ge; ++envc) {
-              uint32_t* img = reinterpret_cast<uint32_t*>(smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)envc * L.rs_env + p.rl.off_avail);
-              for (uint32_t i = lane; i < per_env; i += 32) img[i] = reinterpret_cast<const uint32_t*>(avs)[(uint32_t)envc * per_env + i];
+            const uint32_t inv = 0xFFFFFFFFu / per_env + 1u;  // idx / per_env == umulhi(idx, inv) for idx < 2^16
+            uint8_t* img = smem + L.off_rstage + qslot * L.rs_bytes + p.rl.off_avail;
+            for (uint32_t i = lane; i < (uint32_t)ge * per_env; i += 32) {
+              const uint32_t envc = __umulhi(i, inv);
+              reinterpret_cast<uint32_t*>(img + envc * L.rs_env)[i - envc * per_env] = reinterpret_cast<const uint32_t*>(avs)[i];
             }
           } else {
             const uint32_t per_env = L.av_bytes / 16u;
