@@ -197,7 +197,7 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
   __syncwarp();
 }
 
-template <int NQ>
+template <int NQ, bool PLAIN>  // PLAIN: the word-by-word path of shapes whose per-environment blocks are not 16-byte multiples
 __global__ void __launch_bounds__(TP_THREADS, 1)
     actor_tcp_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TpLayout L) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -525,12 +525,12 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           for (int c = 0; c < nck; ++c) {
             const int ge = min(TP_G, ne - c * TP_G);
             // plain shapes: the image the converters wrote, once they are done with the chunk; else the staged block
-            mbar_wait(L.plain ? &B->cfree[qslot] : &B->full[qslot], qpar, abortf);
+            mbar_wait(PLAIN ? &B->cfree[qslot] : &B->full[qslot], qpar, abortf);
             if (lane < ge) {
               const unsigned long long rec = dstp_s[(kstep & (TP_DST_DEPTH - 1)) * 32 + c * TP_G + lane];
-              const uint8_t* from = L.plain ? smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)lane * L.rs_env
+              const uint8_t* from = PLAIN ? smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)lane * L.rs_env
                                             : stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes;
-              if (rec) bulk_store(reinterpret_cast<void*>(rec), from, L.plain ? L.rs_env : L.obs_bytes);
+              if (rec) bulk_store(reinterpret_cast<void*>(rec), from, PLAIN ? L.rs_env : L.obs_bytes);
             }
             bulk_commit();
             // every lane commits one (possibly empty) group per chunk, so "all but the latest" covers chunk q - 1
@@ -580,7 +580,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const unsigned long long* recs = dstp_s + (it & (TP_DST_DEPTH - 1)) * 32 + c * TP_G;  // this chunk's records
           mbar_wait(&B->full[qslot], qpar, abortf);
           const int items = Rc * L.nchunk;
-          if (L.plain) {
+          if (PLAIN) {
             // rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record image
             for (int j = lane; j < items; j += 32) {
               const int rr = (int)__umulhi((uint32_t)j, inv_nchunk), cc = j - rr * L.nchunk;
@@ -626,7 +626,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             }
           }
           const uint8_t* avs = src + TP_G * L.obs_bytes;  // the chunk's availability bytes, rows contiguous
-          if (L.plain) {
+          if (PLAIN) {
             const uint32_t per_env = L.av_bytes / 4u;  // n A is a multiple of 4
             const uint32_t inv = 0xFFFFFFFFu / per_env + 1u;  // idx / per_env == umulhi(idx, inv) for idx < 2^16
             uint8_t* img = smem + L.off_rstage + qslot * L.rs_bytes + p.rl.off_avail;
@@ -657,7 +657,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             }
             sel[r0 + rc].x = (uint32_t)(bits >> (off & 3u)) & amask;
           }
-          if (L.plain) fence_proxy_async_smem();  // the record image is read by the store warp's bulk stores
+          if (PLAIN) fence_proxy_async_smem();  // the record image is read by the store warp's bulk stores
           __syncwarp();
           if (lane == 0) mbar_arrive(&B->cfree[qslot]);
         }
@@ -936,9 +936,10 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
   if (L.plain && p.E % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
-  auto kernel = L.NQ == 16 ? actor_tcp_kernel<16> : actor_tcp_kernel<32>;
-  static uint32_t configured[2] = {0, 0};
-  uint32_t& conf = configured[L.NQ == 16 ? 0 : 1];
+  auto kernel = L.NQ == 16 ? (L.plain ? actor_tcp_kernel<16, true> : actor_tcp_kernel<16, false>)
+                           : (L.plain ? actor_tcp_kernel<32, true> : actor_tcp_kernel<32, false>);
+  static uint32_t configured[4] = {0, 0, 0, 0};
+  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0)];
   if (L.total > conf) {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return -(int)e;
