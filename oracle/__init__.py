@@ -301,3 +301,39 @@ class Session:
                           C.byref(ts), C.c_int32(0), _ptr(self.counters), C.c_int32(self.n_threads))
         self.t += 1
         return actions, {k: v[0] for k, v in tr.items() if v is not None}
+
+
+TAG_SAMPLE = 5        # Philox stream tag of the learner's episode draws
+SAMPLE_ATTEMPTS = 16  # draws per batch element before it is reported empty
+
+
+def ring_sample(ring: dict, seed: int, draw_index: int, B: int) -> dict:
+    """The learner's draw of B episodes from the replay pool (Algorithm 3: "randomly sample B samples from the
+    experience replay pool"), written out plainly.
+
+    The paper fixes neither the law nor the unit of a sample; the reading taken here: a sample is one complete
+    episode, drawn uniformly and with replacement among the slots whose episode is closed.  Batch element b of
+    draw number `draw_index` makes up to SAMPLE_ATTEMPTS attempts; attempt a takes word 0 of the Philox4x32-10
+    block with counter (draw_index, b, a, TAG_SAMPLE) and key (seed lo, seed hi), proposes slot
+    floor(w0 * C / 2^32) and accepts it if that slot's episode is complete (with at least one step).  An element
+    whose attempts all fail is empty: slot -1, length 0.  The batch is dense, [B][L][...], steps at and beyond
+    an episode's length are zero.
+
+    `ring` holds the pool as arrays indexed [slot][step] (the layout of Session.ring).  Test infrastructure only.
+    """
+    C_, L = ring["obs"].shape[0], ring["obs"].shape[1]
+    out = dict(slot=np.full(B, -1, np.int32), len=np.zeros(B, np.int32), epid=np.full(B, -1, np.int64))
+    for k in ("obs", "avail", "action", "q", "reward", "done"):
+        out[k] = np.zeros((B,) + ring[k].shape[1:], ring[k].dtype)
+    key = (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    for b in range(B):
+        for a in range(SAMPLE_ATTEMPTS):
+            w0 = philox4x32_10((draw_index & 0xFFFFFFFF, b, a, TAG_SAMPLE), key)[0]
+            s = (int(w0) * C_) >> 32
+            if ring["slot_complete"][s] == 1 and ring["slot_len"][s] >= 1:
+                n_steps = int(ring["slot_len"][s])
+                out["slot"][b], out["len"][b], out["epid"][b] = s, n_steps, ring["slot_epid"][s]
+                for k in ("obs", "avail", "action", "q", "reward", "done"):
+                    out[k][b, :n_steps] = ring[k][s, :n_steps]
+                break
+    return out
