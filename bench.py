@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor", "pipelined"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sampler", type=int, default=0, metavar="B",
+                    help="measure the learner-side episode sampler instead: draws of B episodes from a filled ring")
     return ap.parse_args()
 
 
@@ -235,6 +237,45 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sampler(args, cfg, dev):
+    """--sampler B: fills the ring with a rollout long enough to close episodes everywhere, then times draws of B
+    episodes (marl_ring_sample) with CUDA events.  Algorithmic bytes: every sampled record read once, every element
+    of the dense batch written once."""
+    import torch
+    from paper_2205_05248_b200 import binding, workloads
+    cfg = dict(cfg, env=dict(cfg["env"], done_thresh24=int(0.05 * (1 << 24))))   # episodes of about 20 steps
+    weights = workloads.make_weights(cfg)
+    actor = binding.Actor(cfg, device=str(dev), kernel=args.kernel, work_steps=8)
+    actor.set_weights(weights)
+    actor.rollout(cfg["env"], max(cfg["T"], 64), cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+    B, L, n, D, A = args.sampler, cfg["L"], cfg["n"], cfg["D"], cfg["A"]
+    out = None
+    for k in range(args.warmup):
+        out = actor.ring_sample(k, B)
+    torch.cuda.synchronize()
+    lens = out["len"].double()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for k in range(args.steps):
+        actor.ring_sample(1000 + k, B)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    payload = 4 * n * D + n * A + 4 * n + 4 * n * A + 5                     # bytes of one step's fields
+    bytes_per_draw = float(lens.sum()) * payload + B * L * payload + B * 16
+    peaks, peak_kind = load_peaks()
+    achieved = bytes_per_draw / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "episodes/s gathered by marl_ring_sample", "value": B / (ms * 1e-3), "unit": "episodes/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "u8", "data": "synthetic",
+                      "config": {"workload": cfg["name"], "B": B, "L": L, "mean_len": float(lens.mean()),
+                                 "complete_fraction": float((out["slot"] >= 0).double().mean())},
+                      "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
+                                   "kernel": "ring_gather_kernel"}}), flush=True)
+    actor.destroy()
+
+
 def main():
     args = parse_args()
     from paper_2205_05248_b200 import workloads
@@ -251,6 +292,10 @@ def main():
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    if args.sampler > 0:
+        if rank == 0:
+            run_sampler(args, cfg, dev)
+        return
     cfg["seed"] = cfg["seed"] + (rank << 20)          # every rank runs its own replica
     cfg["env"] = dict(cfg["env"], seed=cfg["env"]["seed"] + (rank << 20))
     T, E, n = cfg["T"], cfg["E"], cfg["n"]

@@ -242,6 +242,32 @@ int marl_rollout_noalloc(marl_actor_t* a, const marl_synth_env_t* env, int32_t T
 int marl_actor_set_trace(marl_actor_t* a, int32_t* actions, float* q, int32_t capacity_steps);
 
 int marl_ring_view(const marl_actor_t* a, marl_ring_view_t* out);
+
+/* The learner's read of the pool (Algorithm 3, "randomly sample B samples from the experience replay pool"; the
+ * paper fixes neither the unit nor the law of a sample).  A sample is one complete episode, drawn uniformly and
+ * with replacement among the slots whose episode is closed: batch element b of draw number draw_index makes up to
+ * MARL_SAMPLE_ATTEMPTS attempts; attempt a takes word 0 of the Philox4x32-10 block with counter
+ * (draw_index, b, a, tag 5) and the actor's seed as key, proposes slot floor(w0 * ring_episodes / 2^32) and
+ * accepts it if that slot is complete with at least one step.  An element whose attempts all fail is empty
+ * (slot -1, length 0, id -1).  The episodes are gathered into a dense batch; steps at and beyond an episode's
+ * length are written as zeros.
+ * All pointers are DEVICE arrays owned by the caller, 16-byte aligned, written asynchronously on the actor's
+ * stream and read by nobody else meanwhile; the ring is only read (a rollout enqueued earlier on the same stream
+ * is ordered before the draw).  L = ring_steps. */
+#define MARL_SAMPLE_ATTEMPTS 16
+typedef struct {
+  float* obs;      /* [B][L][n][D] */
+  uint8_t* avail;  /* [B][L][n][A] */
+  int32_t* action; /* [B][L][n] */
+  float* q;        /* [B][L][n][A] */
+  float* reward;   /* [B][L] */
+  uint8_t* done;   /* [B][L] */
+  int32_t* slot;   /* [B] chosen slot or -1 */
+  int32_t* len;    /* [B] steps of the episode (0 if empty) */
+  int64_t* epid;   /* [B] episode id (k * n_envs + e) or -1 */
+} marl_sample_batch_t;
+/* Returns MARL_EINVAL for B < 1 or a NULL field, MARL_EALIGN for a misaligned one, MARL_ECUDA if a launch fails. */
+int marl_ring_sample(marl_actor_t* a, uint32_t draw_index, int32_t B, const marl_sample_batch_t* out);
 int marl_actor_get_state(const marl_actor_t* a, marl_state_view_t* out);
 /* Copies the five device arrays of *in into the actor (device-to-device, on the stream) and sets the step
  * counter.  Together with the ring memory this is a checkpoint. */

@@ -24,7 +24,7 @@ STATUS_NO_AVAIL, STATUS_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4
 EXPORTS = [
     "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_weights_version",
     "marl_actor_step", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
-    "marl_actor_set_trace", "marl_ring_view", "marl_actor_get_state", "marl_actor_set_state",
+    "marl_actor_set_trace", "marl_ring_view", "marl_ring_sample", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
     "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc", "marl_selftest_bounded_wait",
     "marl_measure_ffma_tflops",
@@ -53,6 +53,10 @@ class SynthEnv(C.Structure):
     _fields_ = [("seed", C.c_uint64), ("obs_law", C.c_int32), ("done_thresh24", C.c_uint32),
                 ("avail_thresh_first", C.c_uint32), ("avail_thresh_rest", C.c_uint32), ("avail_split", C.c_int32),
                 ("n_type0", C.c_int32), ("type_block_start", C.c_int32), ("type_block_len", C.c_int32)]
+
+
+class SampleBatch(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("obs", "avail", "action", "q", "reward", "done", "slot", "len", "epid")]
 
 
 class RingView(C.Structure):
@@ -108,6 +112,7 @@ def load_library():
         lib.marl_selftest_bounded_wait.argtypes = [P, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.marl_actor_set_trace.argtypes = [P, P, P, C.c_int32]
         lib.marl_ring_view.argtypes = [P, C.POINTER(RingView)]
+        lib.marl_ring_sample.argtypes = [P, C.c_uint32, C.c_int32, C.POINTER(SampleBatch)]
         lib.marl_actor_get_state.argtypes = [P, C.POINTER(StateView)]
         lib.marl_actor_set_state.argtypes = [P, C.POINTER(StateView)]
         lib.marl_actor_status.argtypes = [P, C.POINTER(C.c_uint32), C.POINTER(Counters)]
@@ -321,6 +326,24 @@ class Actor:
             slot_epid=hdr(v.slot_epid, torch.int64, Cn), slot_len=hdr(v.slot_len, torch.int32, Cn),
             slot_complete=hdr(v.slot_complete, torch.uint8, Cn))
         out["meta"] = {k: getattr(v, k) for k, _ in RingView._fields_}
+        return out
+
+    def ring_sample(self, draw_index: int, B: int) -> dict:
+        """marl_ring_sample into fresh device tensors: a dense batch of B episodes drawn from the ring."""
+        c = self.cfg
+        L, n, D, A = c["L"], c["n"], c["D"], c["A"]
+        dev = self.device
+        out = dict(obs=torch.empty((B, L, n, D), dtype=torch.float32, device=dev),
+                   avail=torch.empty((B, L, n, A), dtype=torch.uint8, device=dev),
+                   action=torch.empty((B, L, n), dtype=torch.int32, device=dev),
+                   q=torch.empty((B, L, n, A), dtype=torch.float32, device=dev),
+                   reward=torch.empty((B, L), dtype=torch.float32, device=dev),
+                   done=torch.empty((B, L), dtype=torch.uint8, device=dev),
+                   slot=torch.empty((B,), dtype=torch.int32, device=dev),
+                   len=torch.empty((B,), dtype=torch.int32, device=dev),
+                   epid=torch.empty((B,), dtype=torch.int64, device=dev))
+        sb = SampleBatch(*[_dptr(out[k]) for k, _ in SampleBatch._fields_])
+        _check(self.lib.marl_ring_sample(self.handle, C.c_uint32(draw_index), C.c_int32(B), C.byref(sb)))
         return out
 
     def get_state(self) -> dict:

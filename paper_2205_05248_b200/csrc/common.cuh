@@ -66,6 +66,20 @@ struct ActorParams {
   uint32_t* status;
 };
 
+// Everything the episode sampler needs (ring_sample.cu).  Passed by value.
+struct SampleParams {
+  int32_t B, C, L, n, D, A, E;
+  uint64_t seed;
+  uint32_t draw_index;
+  const uint8_t* ring;
+  RecordLayout rl;
+  long long slot_stride;
+  const long long* slot_epid;
+  const int32_t* slot_len;
+  const uint8_t* slot_complete;
+  marl_sample_batch_t out;
+};
+
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
                                               uint32_t k1, uint32_t out[4]) {
 #pragma unroll

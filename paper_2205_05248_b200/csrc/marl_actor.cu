@@ -28,6 +28,7 @@ void tc_tiling(int E, int n, int sms, int* ept, int* num_tiles);
 int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream);
 bool tcp_supported(int n, int D, int A, int H, int prec);
 int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream);
+int launch_ring_sample(const SampleParams& p, cudaStream_t stream);
 }  // namespace marl
 
 using namespace marl;
@@ -582,6 +583,33 @@ int marl_ring_view(const marl_actor_t* a, marl_ring_view_t* out) {
   out->slot_epid = reinterpret_cast<int64_t*>(a->ring + a->ro.epid);
   out->slot_len = reinterpret_cast<int32_t*>(a->ring + a->ro.len);
   out->slot_complete = a->ring + a->ro.complete;
+  return MARL_OK;
+}
+
+int marl_ring_sample(marl_actor_t* a, uint32_t draw_index, int32_t B, const marl_sample_batch_t* out) {
+  if (!a || !out) return fail(MARL_EINVAL, "actor or out is NULL");
+  if (B < 1 || B > 65535) return fail(MARL_EINVAL, "B must be in 1 .. 65535");
+  const void* ptrs[9] = {out->obs, out->avail, out->action, out->q, out->reward, out->done, out->slot, out->len, out->epid};
+  for (const void* q : ptrs) {
+    if (!q) return fail(MARL_EINVAL, "a field of the batch is NULL");
+    if (reinterpret_cast<uintptr_t>(q) % 16) return fail(MARL_EALIGN, "the fields of the batch must be 16-byte aligned");
+  }
+  const marl_actor_config_t& c = a->cfg;
+  marl::SampleParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = B; p.C = c.ring_episodes; p.L = c.ring_steps; p.n = c.n_agents; p.D = c.obs_dim; p.A = c.n_actions; p.E = c.n_envs;
+  p.seed = c.seed;
+  p.draw_index = draw_index;
+  p.ring = a->ring + a->ro.records;
+  p.rl = a->rl;
+  p.slot_stride = (long long)c.ring_steps * a->rl.rec_bytes;
+  p.slot_epid = reinterpret_cast<const long long*>(a->ring + a->ro.epid);
+  p.slot_len = reinterpret_cast<const int32_t*>(a->ring + a->ro.len);
+  p.slot_complete = a->ring + a->ro.complete;
+  p.out = *out;
+  const int rc = marl::launch_ring_sample(p, a->stream);
+  if (rc < 0) return fail(MARL_ECUDA, "sampler kernel launch: %s", cudaGetErrorString((cudaError_t)(-rc)));
+  a->launches += (uint64_t)rc;
   return MARL_OK;
 }
 
