@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--H", type=int, default=None)
     ap.add_argument("--precision", default=None, choices=[None, "fp32", "bf16"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor", "pipelined"])
+    ap.add_argument("--refresh", action="store_true",
+                    help="publish a new network during every step, effective at the middle of the next rollout "
+                         "(the learner's model update running beside the workers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sampler", type=int, default=0, metavar="B",
@@ -307,8 +310,15 @@ def main():
     input_bytes = sum(t.numel() * t.element_size() for t in staged)
     torch.cuda.synchronize()
 
+    nets = [weights, workloads.make_weights(cfg, seed=cfg["seed"] + 1)]
+    done_steps = [0]
+
     def one_step():
+        if args.refresh:
+            k = done_steps[0] // T + 1
+            actor.publish_weights(nets[k % 2], version=k + 1, effective_step=done_steps[0] + T // 2)
         actor.rollout_staged(*staged, T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+        done_steps[0] += T
 
     for _ in range(args.warmup):
         one_step()
@@ -339,10 +349,11 @@ def main():
     value = world * agent_steps / (ms_total * 1e-3)
 
     peaks, peak_kind = load_peaks()
-    kernel_ms = ms_local / max(launches, 1)            # one actor kernel per bench step
-    bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T) * E * n * T
+    kernel_ms = ms_local / max(launches, 1)            # one actor kernel per bench step (two when it is split)
+    T_launch = T * args.steps / max(launches, 1)       # environment steps one launch covers
+    bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T_launch) * E * n * T_launch
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
-    flop_rate = flops_per_agent_step(cfg) * E * n * T / (kernel_ms * 1e-3) / 1e12
+    flop_rate = flops_per_agent_step(cfg) * E * n * T_launch / (kernel_ms * 1e-3) / 1e12
     kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel"}.get(actor.kernel_name, "actor_ffma_kernel")
     if cfg["precision"] == "fp32":
         # the fp32 path is bound by plain FFMA arithmetic: peak measured on this device by the library's FMA loop
@@ -353,9 +364,9 @@ def main():
                     "hbm_gbs_achieved": achieved}
     else:
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": measured_traffic(kname, E * n * T),
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": measured_traffic(kname, E * n * T_launch),
                     "peak_source": peak_kind, "kernel": kname,
-                    "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T),
+                    "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T_launch),
                     "tflops_effective": flop_rate}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -366,6 +377,9 @@ def main():
                        "step": f"one marl_rollout_staged call = T={T} environment steps over E={E} environments",
                        "l2": f"inputs larger than L2 ({input_bytes / 1e6:.0f} MB staged per step, read once)"},
             "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline}
+    if args.refresh:
+        line["config"]["weight_refresh"] = (f"one publication per step, effective {T // 2} environment steps into the "
+                                            f"rollout (the launch is split there); final version {actor.weights_version}")
 
     # ---- end to end through the host-buffer entry point: H2D of each step's inputs, D2H of its actions ----
     if not args.no_e2e:

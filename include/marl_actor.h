@@ -181,6 +181,19 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out);
 int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
                            const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
                            const float* b2, uint64_t version);
+
+/* The learner's refresh of the shared model while the workers run (Sec. III-B: the learner updates the model in
+ * the shared memory pool; Algorithm 2: a worker gets the parameters at the start of an iteration).  The network
+ * (HOST arrays as for marl_actor_set_weights, copied before the call returns) becomes the one in use from global
+ * step effective_step on (>= the number of steps enqueued so far): the upload runs on a stream of its own beside
+ * the steps already enqueued, into the second of two weight images; a later call that spans effective_step runs
+ * the steps before it on the old image, makes the stream wait for the upload, swaps the images and runs the rest
+ * on the new one - deterministic, whatever the timing.  One publication can be pending: a newer one replaces it,
+ * marl_actor_set_weights drops it.  marl_actor_weights_version reports the version of the image in use by the next
+ * step to be enqueued. */
+int marl_actor_publish_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
+                               const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
+                               const float* b2, uint64_t version, uint64_t effective_step);
 uint64_t marl_actor_weights_version(const marl_actor_t* a);
 
 /* One decision step for all E environments (Algorithm 2, loop body) with recording (Algorithm 1).

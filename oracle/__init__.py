@@ -238,6 +238,11 @@ class Session:
         lib().oracle_init(C.byref(self._d), _ptr(self.env_ids), C.c_int32(Es), C.byref(st),
                           C.byref(rg) if rg is not None else None)
 
+    def set_weights(self, weights: dict):
+        """The shared model after a learner update (Sec. III-B): used by every later step."""
+        self.weights = weights
+        self._w, self._wkeep = _weights_struct(weights)
+
     def _structs(self):
         st = _State(_ptr(self.h), _ptr(self.last_action), _ptr(self.slot), _ptr(self.pos), _ptr(self.ep_count))
         rg = None

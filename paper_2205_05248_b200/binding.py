@@ -22,7 +22,8 @@ KERNEL = {"auto": 0, "ffma": 1, "tensor": 2, "pipelined": 3}
 STATUS_NO_AVAIL, STATUS_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4
 
 EXPORTS = [
-    "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_weights_version",
+    "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_publish_weights",
+    "marl_actor_weights_version",
     "marl_actor_step", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
     "marl_actor_set_trace", "marl_ring_view", "marl_ring_sample", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
@@ -102,6 +103,7 @@ def load_library():
         lib.marl_actor_query_sizes.argtypes = [C.POINTER(Config), C.POINTER(Sizes)]
         lib.marl_actor_create.argtypes = [C.POINTER(Config), C.POINTER(P)]
         lib.marl_actor_set_weights.argtypes = [P] + [P] * 8 + [C.c_uint64]
+        lib.marl_actor_publish_weights.argtypes = [P] + [P] * 8 + [C.c_uint64, C.c_uint64]
         lib.marl_actor_step.argtypes = [P, P, P, P, P, C.c_float, P]
         lib.marl_actor_step_host.argtypes = [P, P, P, P, P, C.c_float, P]
         lib.marl_env_generate.argtypes = [P, C.POINTER(SynthEnv), C.c_uint32, C.c_int32, P, P, P, P]
@@ -224,6 +226,18 @@ class Actor:
                 for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")]
         _check(self.lib.marl_actor_set_weights(self.handle, *[a.ctypes.data_as(C.c_void_p) for a in arrs],
                                                C.c_uint64(version)))
+
+    def publish_weights(self, w: dict, version: int, effective_step: int):
+        """marl_actor_publish_weights: the network in use from global step effective_step on."""
+        import numpy as np
+        arrs = [np.ascontiguousarray(w[k], dtype=np.float32)
+                for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")]
+        _check(self.lib.marl_actor_publish_weights(self.handle, *[a.ctypes.data_as(C.c_void_p) for a in arrs],
+                                                   C.c_uint64(version), C.c_uint64(effective_step)))
+
+    @property
+    def weights_version(self) -> int:
+        return int(self.lib.marl_actor_weights_version(self.handle))
 
     # -- stepping ---------------------------------------------------------------------------------
     def step(self, obs, avail, reward, done, eps: float, actions_out=None):

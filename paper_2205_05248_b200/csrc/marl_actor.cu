@@ -80,7 +80,7 @@ static FfmaWeightOffsets ffma_weight_offsets(int n, int D, int A, int H) {
   return w;
 }
 
-struct StateOffsets { size_t h, last_action, slot, pos, ep_count, counters, status, wff, wpack, total; };
+struct StateOffsets { size_t h, last_action, slot, pos, ep_count, counters, status, wff[2], wpack[2], total; };  // two weight images
 struct RingOffsets { size_t records, epid, len, complete, total; };
 struct WorkOffsets { size_t obs, avail, reward, done, actions, total; };
 
@@ -110,8 +110,10 @@ static StateOffsets state_offsets(const marl_actor_config_t& c) {
   s.ep_count = cv.take(sizeof(int64_t) * c.n_envs);
   s.counters = cv.take(sizeof(uint64_t) * CNT_N);
   s.status = cv.take(sizeof(uint32_t) * 4);
-  s.wff = cv.take(ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
-  s.wpack = cv.take(tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden));
+  for (int i = 0; i < 2; ++i) {
+    s.wff[i] = cv.take(ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
+    s.wpack[i] = cv.take(tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden));
+  }
   s.total = cv.off;
   return s;
 }
@@ -181,6 +183,13 @@ struct marl_actor {
   int32_t trace_cap, trace_next;
   uint64_t launches;
   std::vector<uint8_t> host_pack;
+  // weight publication: the image in use, the copy stream, and the publication waiting for its step
+  int wslot;
+  cudaStream_t copy_stream;
+  cudaEvent_t upload_done, image_free;
+  bool image_free_recorded, pending;
+  uint64_t pending_version, pending_step;
+  uint8_t* host_pack2;  // pinned, so that the upload really runs beside the steps
 };
 
 __global__ void init_state_kernel(int E, int n, int H, int S, int C, float* h, int32_t* la, int32_t* slot,
@@ -268,6 +277,12 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   a->trace_q = nullptr;
   a->trace_cap = a->trace_next = 0;
   a->launches = 0;
+  a->wslot = 0;
+  a->host_pack2 = nullptr;
+  a->copy_stream = nullptr;
+  a->upload_done = a->image_free = nullptr;
+  a->image_free_recorded = a->pending = false;
+  a->pending_version = a->pending_step = 0;
 
   const bool tc_ok = tc_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
   const bool tcp_ok = tcp_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
@@ -320,6 +335,13 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
 void marl_actor_destroy(marl_actor_t* a) {
   if (!a) return;
   cudaStreamSynchronize(a->stream);
+  if (a->copy_stream) {
+    cudaStreamSynchronize(a->copy_stream);
+    cudaStreamDestroy(a->copy_stream);
+    cudaEventDestroy(a->upload_done);
+    cudaEventDestroy(a->image_free);
+    cudaFreeHost(a->host_pack2);
+  }
   if (a->own_ring) cudaFree(a->ring);
   if (a->own_state) cudaFree(a->state);
   if (a->own_work) cudaFree(a->work);
@@ -336,19 +358,16 @@ static float to_bf16_value(float v) {
   return v;
 }
 
-int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
-                           const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
-                           const float* b2, uint64_t version) {
-  if (!a) return fail(MARL_EINVAL, "actor is NULL");
-  if (!W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a weight pointer is NULL");
+// Packs the network into `dst` as the kernels read it: the FFMA image (k-major fp32, bf16-representable values in
+// the bf16 precision) followed by the tensor-core image.
+static void pack_weights_host(marl_actor* a, const float* W1, const float* b1, const float* W_ih, const float* b_ih,
+                              const float* W_hh, const float* b_hh, const float* W2, const float* b2,
+                              uint8_t* hp) {
   const int n = a->cfg.n_agents, D = a->cfg.obs_dim, A = a->cfg.n_actions, H = a->cfg.hidden;
   const int I = D + n + A;
   const bool lowp = a->cfg.precision == MARL_PRECISION_BF16;
   const size_t tcb = tc_wpack_bytes(n, D, A, H);
-  // The previous upload may still be in flight from this staging buffer.
-  CU_TRY(cudaStreamSynchronize(a->stream));
-  a->host_pack.assign(a->wo.total + tcb, 0);
-  uint8_t* hp = a->host_pack.data();
+  memset(hp, 0, a->wo.total + tcb);
   auto q = [lowp](float v) { return lowp ? to_bf16_value(v) : v; };
   float* W1T = reinterpret_cast<float*>(hp + a->wo.W1T);
   for (int j = 0; j < H; ++j)
@@ -366,14 +385,64 @@ int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, co
   memcpy(hp + a->wo.bih, b_ih, sizeof(float) * 3 * H);
   memcpy(hp + a->wo.bhh, b_hh, sizeof(float) * 3 * H);
   memcpy(hp + a->wo.b2, b2, sizeof(float) * A);
-  CU_TRY(cudaMemcpyAsync(a->state + a->so.wff, hp, a->wo.total, cudaMemcpyHostToDevice, a->stream));
-  if (tcb && (tc_supported(n, D, A, H, a->cfg.precision) || tcp_supported(n, D, A, H, a->cfg.precision))) {
+  if (tcb && (tc_supported(n, D, A, H, a->cfg.precision) || tcp_supported(n, D, A, H, a->cfg.precision)))
     tc_pack_weights(n, D, A, H, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, hp + a->wo.total);
-    CU_TRY(cudaMemcpyAsync(a->state + a->so.wpack, hp + a->wo.total, tcb, cudaMemcpyHostToDevice, a->stream));
+}
+
+static int upload_weights(marl_actor* a, const uint8_t* src, int image, cudaStream_t stream) {
+  const marl_actor_config_t& c = a->cfg;
+  const size_t tcb = tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden);
+  CU_TRY(cudaMemcpyAsync(a->state + a->so.wff[image], src, a->wo.total, cudaMemcpyHostToDevice, stream));
+  if (tcb) CU_TRY(cudaMemcpyAsync(a->state + a->so.wpack[image], src + a->wo.total, tcb, cudaMemcpyHostToDevice, stream));
+  return MARL_OK;
+}
+
+int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
+                           const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
+                           const float* b2, uint64_t version) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a weight pointer is NULL");
+  // The previous upload may still be in flight from this staging buffer, and enqueued steps may still read the image.
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  if (a->pending) {  // a publication that has not taken effect is dropped
+    CU_TRY(cudaStreamSynchronize(a->copy_stream));
+    a->pending = false;
   }
+  a->host_pack.resize(a->wo.total + tc_wpack_bytes(a->cfg.n_agents, a->cfg.obs_dim, a->cfg.n_actions, a->cfg.hidden));
+  pack_weights_host(a, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, a->host_pack.data());
+  const int rc = upload_weights(a, a->host_pack.data(), a->wslot, a->stream);
+  if (rc) return rc;
   CU_TRY(cudaStreamSynchronize(a->stream));
   a->weights_version = version;
   a->have_weights = true;
+  return MARL_OK;
+}
+
+int marl_actor_publish_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
+                               const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
+                               const float* b2, uint64_t version, uint64_t effective_step) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a weight pointer is NULL");
+  if (!a->have_weights) return fail(MARL_EINVAL, "marl_actor_set_weights has not been called");
+  if (effective_step < a->step) return fail(MARL_EINVAL, "effective_step %llu is already enqueued (next step is %llu)",
+                                            (unsigned long long)effective_step, (unsigned long long)a->step);
+  if (!a->copy_stream) {
+    CU_TRY(cudaStreamCreateWithFlags(&a->copy_stream, cudaStreamNonBlocking));
+    CU_TRY(cudaEventCreateWithFlags(&a->upload_done, cudaEventDisableTiming));
+    CU_TRY(cudaEventCreateWithFlags(&a->image_free, cudaEventDisableTiming));
+    CU_TRY(cudaMallocHost(&a->host_pack2, a->wo.total + tc_wpack_bytes(a->cfg.n_agents, a->cfg.obs_dim, a->cfg.n_actions, a->cfg.hidden)));
+  }
+  // an earlier publication's copy reads host_pack2 and writes the same image: let it finish (it is replaced)
+  CU_TRY(cudaStreamSynchronize(a->copy_stream));
+  pack_weights_host(a, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, a->host_pack2);
+  // the idle image was last read by steps enqueued before the previous switch
+  if (a->image_free_recorded) CU_TRY(cudaStreamWaitEvent(a->copy_stream, a->image_free, 0));
+  const int rc = upload_weights(a, a->host_pack2, a->wslot ^ 1, a->copy_stream);
+  if (rc) return rc;
+  CU_TRY(cudaEventRecord(a->upload_done, a->copy_stream));
+  a->pending = true;
+  a->pending_version = version;
+  a->pending_step = effective_step;
   return MARL_OK;
 }
 
@@ -389,7 +458,7 @@ static void fill_params(marl_actor* a, ActorParams& p) {
   p.prec = c.precision;
   p.seed = c.seed;
   uint8_t* st = a->state;
-  const uint8_t* w = st + a->so.wff;
+  const uint8_t* w = st + a->so.wff[a->wslot];
   p.W1T = reinterpret_cast<const float*>(w + a->wo.W1T);
   p.b1 = reinterpret_cast<const float*>(w + a->wo.b1);
   p.WihT = reinterpret_cast<const float*>(w + a->wo.WihT);
@@ -398,7 +467,7 @@ static void fill_params(marl_actor* a, ActorParams& p) {
   p.bhh = reinterpret_cast<const float*>(w + a->wo.bhh);
   p.W2 = reinterpret_cast<const float*>(w + a->wo.W2);
   p.b2 = reinterpret_cast<const float*>(w + a->wo.b2);
-  p.wpack = st + a->so.wpack;
+  p.wpack = st + a->so.wpack[a->wslot];
   p.h = reinterpret_cast<float*>(st + a->so.h);
   p.last_action = reinterpret_cast<int32_t*>(st + a->so.last_action);
   p.slot = reinterpret_cast<int32_t*>(st + a->so.slot);
@@ -425,6 +494,26 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   if (!a->have_weights) return fail(MARL_EINVAL, "marl_actor_set_weights has not been called");
   if (a->step + (uint64_t)T > 0xFFFFFFFFull) return fail(MARL_EINVAL, "step counter would exceed 32 bits");
   const marl_actor_config_t& c = a->cfg;
+  if (a->pending && a->step + (uint64_t)T > a->pending_step) {
+    // A published network takes effect inside this span: the steps before it run on the current image, then the
+    // stream waits for the upload (which has been running beside the earlier steps) and the images are swapped.
+    const int T1 = (int)(a->pending_step - a->step);
+    if (T1 > 0) {
+      const int rc1 = enqueue_steps(a, obs, avail, reward, done, T1, eps_const, eps, eps_start, eps_end, anneal, nullptr);
+      if (rc1) return rc1;
+      obs += (size_t)T1 * c.n_envs * c.n_agents * c.obs_dim;
+      avail += (size_t)T1 * c.n_envs * c.n_agents * c.n_actions;
+      reward += (size_t)T1 * c.n_envs;
+      done += (size_t)T1 * c.n_envs;
+      T -= T1;
+    }
+    CU_TRY(cudaStreamWaitEvent(a->stream, a->upload_done, 0));
+    CU_TRY(cudaEventRecord(a->image_free, a->stream));  // the image in use so far is idle once the work above is done
+    a->image_free_recorded = true;
+    a->wslot ^= 1;
+    a->weights_version = a->pending_version;
+    a->pending = false;
+  }
   ActorParams p;
   fill_params(a, p);
   p.T = T;

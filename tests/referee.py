@@ -52,8 +52,10 @@ def run_gpu_rollout(cfg, weights, kernel="auto", T=None, splits=None, want_q=Tru
     return actor, acts, q
 
 
-def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=None, n_threads=None):
-    """Checks parts 1-4 for the listed environments (default: all).  Returns a summary dict."""
+def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=None, n_threads=None,
+            weight_schedule=()):
+    """Checks parts 1-4 for the listed environments (default: all).  Returns a summary dict.
+    weight_schedule: (step, weights) pairs in rising step order; the oracle switches to that network at that step."""
     T = cfg["T"] if T is None else T
     E, n, A, H = cfg["E"], cfg["n"], cfg["A"], cfg["H"]
     ids = np.arange(E) if env_ids is None else np.asarray(env_ids)
@@ -65,7 +67,15 @@ def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_
     g_q = gpu_q[:T].index_select(1, tids).cpu().numpy()
 
     sess = oracle.Session(cfg, weights, ids, n_threads=n_threads or oracle.hardware_threads())
-    tr = sess.rollout(cfg["env"], T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], adopt=g_act)
+    cuts = [0] + [int(s0) for s0, _ in weight_schedule] + [T]
+    parts = []
+    for k in range(len(cuts) - 1):
+        if k:
+            sess.set_weights(weight_schedule[k - 1][1])
+        if cuts[k + 1] > cuts[k]:
+            parts.append(sess.rollout(cfg["env"], cuts[k + 1] - cuts[k], cfg["eps_start"], cfg["eps_end"],
+                                      cfg["anneal_steps"], adopt=g_act[cuts[k]:cuts[k + 1]]))
+    tr = {key: np.concatenate([part[key] for part in parts]) for key in parts[0]}
 
     # ---- part 2: the GPU's decision follows from its own Q row ----
     eps = eps_schedule(cfg, 0, T)

@@ -177,3 +177,25 @@ def test_adopted_actions_feed_back_and_are_recorded():
     assert not np.array_equal(tf["q"][3, 1, 0], tr["q"][3, 1, 0])
     assert np.array_equal(tf["q"][3, 0], tr["q"][3, 0])        # the other environment is untouched
     assert forced.ring["action"][forced.slot[1], 2, 0] == adopt[2, 1, 0]
+
+
+def test_weight_switch_uses_the_new_network_from_the_next_step():
+    """Sec. III-B: workers act with whatever model the learner last placed in the shared pool.  After a switch the
+    Q rows are those of the new network applied (by the single-agent forward) to the carried-over hidden state."""
+    cfg = workloads.small_config(E=3, C=6, L=5, T=9, env=dict(done_thresh24=0))
+    sess, w0 = _session(cfg)
+    w1 = workloads.make_weights(cfg, seed=cfg["seed"] + 5)
+    t1 = _roll(sess, cfg, T=4)
+    h_before, la_before = sess.h.copy(), sess.last_action.copy()
+    sess.set_weights(w1)
+    t2 = _roll(sess, cfg, T=1)
+    for x in range(cfg["E"]):
+        for i in range(cfg["n"]):
+            q_new, _ = oracle.agent_forward(cfg, w1, t2["obs"][0, x, i], i, int(la_before[x, i]), h_before[x, i])
+            q_old, _ = oracle.agent_forward(cfg, w0, t2["obs"][0, x, i], i, int(la_before[x, i]), h_before[x, i])
+            assert np.allclose(t2["q"][0, x, i], q_new, rtol=1e-6, atol=1e-7)
+            assert not np.allclose(t2["q"][0, x, i], q_old, rtol=1e-3, atol=1e-4)
+    # the steps before the switch are those of a session that never switched
+    plain, _ = _session(cfg)
+    t0 = _roll(plain, cfg, T=4)
+    assert all(np.array_equal(t0[k], t1[k]) for k in t0)
