@@ -203,6 +203,20 @@ uint64_t marl_actor_weights_version(const marl_actor_t* a);
 int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,
                     const uint8_t* done, float eps, int32_t* actions_out);
 
+/* The step for the environments that have an observation ready (the actors interact with their environments
+ * asynchronously, Sec. III-A; the worker serves the observations that have arrived, Algorithm 2): only the M
+ * listed environments decide, record and advance; the state and the ring slots of the others are untouched.
+ * env_ids i32[M] is a HOST array (the host knows which pipes hold data), copied before the call returns; every
+ * entry in [0, E), none twice (MARL_EINVAL otherwise, nothing enqueued).  The other arrays are DEVICE arrays, dense
+ * over the list: row x belongs to environment env_ids[x]: obs f32[M][n][D], avail u8[M][n][A], reward f32[M],
+ * done u8[M], actions_out i32[M][n] (may be NULL).  The call consumes one index of the global step counter, which
+ * keys the exploration stream as (seed, step, environment, agent) with the environment's own index; a trace row
+ * of this step is written at the environment's own index as well.  Runs on the CUDA-core kernel for every shape
+ * and precision. */
+int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
+                           const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
+                           int32_t* actions_out);
+
 /* The same step with HOST buffers (the observation-action pipe of Algorithms 1 and 2 when the simulators
  * run on the host): copies the four inputs to the device, runs the step, copies the actions back and
  * SYNCHRONISES the stream before returning.  Pinned host memory makes the copies asynchronous. */

@@ -252,9 +252,9 @@ class Session:
                                               "slot_len", "slot_complete")])
         return st, rg
 
-    def _alloc_trace(self, T, want):
+    def _alloc_trace(self, T, want, rows=None):
         c = self.cfg
-        Es, n, D, A, H = len(self.env_ids), c["n"], c["D"], c["A"], c["H"]
+        Es, n, D, A, H = (len(self.env_ids) if rows is None else rows), c["n"], c["D"], c["A"], c["H"]
         shapes = dict(obs=((T, Es, n, D), np.float32), avail=((T, Es, n, A), np.uint8),
                       reward=((T, Es), np.float32), done=((T, Es), np.uint8), q=((T, Es, n, A), np.float32),
                       h=((T, Es, n, H), np.float32), action=((T, Es, n), np.int32),
@@ -304,6 +304,46 @@ class Session:
                           C.c_uint32(self.t), C.c_float(eps), _ptr(obs), _ptr(avail), _ptr(reward), _ptr(done),
                           _ptr(adopt), C.byref(st), C.byref(rg) if rg is not None else None, _ptr(actions),
                           C.byref(ts), C.c_int32(0), _ptr(self.counters), C.c_int32(self.n_threads))
+        self.t += 1
+        return actions, {k: v[0] for k, v in tr.items() if v is not None}
+
+    def step_subset(self, env_ids, obs, avail, reward, done, eps: float, adopt=None, trace=()):
+        """One decision step for the listed environments only (actors are asynchronous, Sec. III-A: the worker
+        serves the observations that have arrived).  Index plumbing around the same step routine: the listed rows of
+        the state and of the pool image are copied out, stepped with the session's step counter, and copied back;
+        every other row is untouched.  Returns (actions [M][n], traces)."""
+        c = self.cfg
+        ids = _c(env_ids, np.int32)
+        M, n, S = len(ids), c["n"], self.S
+        where = {int(e): x for x, e in enumerate(self.env_ids)}
+        loc = np.array([where[int(e)] for e in ids], np.int64)
+        assert len(set(loc.tolist())) == M, "an environment is listed twice"
+        obs = _c(obs, np.float32)
+        avail = _c(avail, np.uint8)
+        reward = _c(reward, np.float32)
+        done = _c(done, np.uint8)
+        assert obs.shape == (M, n, c["D"]) and avail.shape == (M, n, c["A"]) and reward.shape == (M,)
+        if adopt is not None:
+            adopt = _c(adopt, np.int32)
+        sub = {k: np.ascontiguousarray(getattr(self, k)[loc]) for k in ("h", "last_action", "slot", "pos", "ep_count")}
+        st = _State(*[_ptr(sub[k]) for k in ("h", "last_action", "slot", "pos", "ep_count")])
+        rg, rsub = None, None
+        if self.ring is not None:
+            names = ("obs", "avail", "action", "q", "reward", "done", "slot_epid", "slot_len", "slot_complete")
+            rows = (loc[:, None] * S + np.arange(S)[None, :]).reshape(-1)       # pool rows of the listed environments
+            rsub = {k: np.ascontiguousarray(self.ring[k][rows]) for k in names}
+            rg = _Ring(*[_ptr(rsub[k]) for k in names])
+        tr, ts = self._alloc_trace(1, set(trace or ()), rows=M)
+        actions = np.zeros((M, n), np.int32)
+        lib().oracle_step(C.byref(self._d), C.byref(self._w), _ptr(ids), C.c_int32(M), C.c_uint32(self.t),
+                          C.c_float(eps), _ptr(obs), _ptr(avail), _ptr(reward), _ptr(done), _ptr(adopt), C.byref(st),
+                          C.byref(rg) if rg is not None else None, _ptr(actions), C.byref(ts), C.c_int32(0),
+                          _ptr(self.counters), C.c_int32(self.n_threads))
+        for k, v in sub.items():
+            getattr(self, k)[loc] = v
+        if rsub is not None:
+            for k, v in rsub.items():
+                self.ring[k][rows] = v
         self.t += 1
         return actions, {k: v[0] for k, v in tr.items() if v is not None}
 

@@ -47,7 +47,7 @@ __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H)
   s.off_qs = o; o += sizeof(float) * FF_RMAX * FF_QSTRIDE;
   s.off_mask = o; o += sizeof(uint32_t) * FF_RMAX;
   s.off_la = o; o += sizeof(int32_t) * FF_RMAX;
-  s.off_env = o; o += 32 * FF_RMAX;  // per-environment scratch: see EnvSlot
+  s.off_env = o; o += 40 * FF_RMAX;  // per-environment scratch: see EnvSlot
   s.off_w = o;
   s.w_floats = ffma_weight_floats(n, D, A, H);
   s.wsmem = (o + sizeof(float) * s.w_floats <= 227 * 1024) ? 1 : 0;  // resident weights if they fit
@@ -56,14 +56,17 @@ __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H)
   return s;
 }
 
-struct EnvSlot {            // 32 bytes per environment of the tile
+struct EnvSlot {            // 40 bytes per environment of the tile
   long long epc;
+  int32_t eid;              // the environment's index in the actor (not in the call)
   int32_t slot, pos;
   float reward;
   int32_t done;             // this step's done flag
   int32_t ok;               // cursor was in range at tile load
   int32_t reset;            // episode closed this step
 };
+
+static_assert(sizeof(EnvSlot) == 40, "the shared-memory plan reserves 40 bytes per environment");
 
 __device__ __forceinline__ float sigmoid_accurate(float x) { return 1.0f / (1.0f + expf(-x)); }
 
@@ -125,7 +128,9 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
 
   for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
     const int e0 = tile * p.ept;
-    const int ne = min(p.ept, p.E - e0);  // environments in this tile
+    const int ne = min(p.ept, p.M - e0);  // environments in this tile (e0 counts the call's rows)
+    // the environment behind row-of-the-call x: x itself, or the caller's list for a partial step
+    auto env_of = [&](int x) { return p.env_ids ? __ldg(p.env_ids + x) : x; };
     const int R = ne * n;                 // live rows
     int cur = 0;
     auto prefetch_obs = [&](int s) {
@@ -142,15 +147,17 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
     // ---- tile load: hidden state, last actions, ring cursors ----
     for (int idx = tid; idx < R * H; idx += FF_THREADS) {
       const int r = idx / H, j = idx - r * H;
-      const float v = p.h[(size_t)e0 * n * H + idx];
+      const int el = r / n;
+      const float v = p.h[((size_t)env_of(e0 + el) * n + (r - el * n)) * H + j];
       hs[r * Hp + j] = v;
     }
-    for (int r = tid; r < FF_RMAX; r += FF_THREADS) la[r] = (r < R) ? p.last_action[e0 * n + r] : -1;
+    for (int r = tid; r < FF_RMAX; r += FF_THREADS) la[r] = (r < R) ? p.last_action[env_of(e0 + r / n) * n + r % n] : -1;
     if (tid < ne) {
       EnvSlot s;
-      s.slot = p.slot[e0 + tid];
-      s.pos = p.pos[e0 + tid];
-      s.epc = p.ep_count[e0 + tid];
+      s.eid = env_of(e0 + tid);
+      s.slot = p.slot[s.eid];
+      s.pos = p.pos[s.eid];
+      s.epc = p.ep_count[s.eid];
       s.reward = 0.f;
       s.done = 0;
       s.reset = 0;
@@ -220,7 +227,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           es.done = p.done[(size_t)s * p.env_step_stride + e0 + tid] ? 1 : 0;
           es.reset = 0;
           if (es.ok && es.pos == 0) {  // an episode opens in this slot
-            p.slot_epid[es.slot] = es.epc * (long long)p.E + (e0 + tid);
+            p.slot_epid[es.slot] = es.epc * (long long)p.E + es.eid;
             p.slot_len[es.slot] = 0;
             p.slot_complete[es.slot] = 0;
           }
@@ -378,7 +385,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       // ---- phase E: choice and recording, one thread per row ----
       if (tid < R) {
         const int el = tid / n, ai = tid - el * n;
-        const int e = e0 + el;
+        const int e = envs[el].eid;
         const float* qrow = qs + tid * FF_QSTRIDE;
         uint32_t flags;
         const int act = select_action([&](int a) { return qrow[a]; }, A, masks[tid], eps, p.seed, t,
@@ -401,7 +408,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           if (p.trace_q)
             for (int a = 0; a < A; ++a) p.trace_q[grow * A + a] = qrow[a];
         }
-        if (p.actions_out && s == p.T - 1) p.actions_out[(size_t)e * n + ai] = act;
+        if (p.actions_out && s == p.T - 1) p.actions_out[(size_t)(e0 + el) * n + ai] = act;
       }
       __syncthreads();  // the rows above read the cursors that the environment threads advance below
       // ---- phase F (first half): reward/done and the episode cursor, one thread per environment ----
@@ -418,7 +425,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             c_episodes += 1;
             if (!es.done) c_trunc += 1;
             es.epc += 1;
-            es.slot = (e0 + tid) * p.S + (int)(es.epc % p.S);
+            es.slot = es.eid * p.S + (int)(es.epc % p.S);
             es.pos = 0;
             es.reset = 1;
           } else {
@@ -442,15 +449,16 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
     // ---- tile store ----
     for (int idx = tid; idx < R * H; idx += FF_THREADS) {
       const int r = idx / H, j = idx - r * H;
-      p.h[(size_t)e0 * n * H + idx] = hs[cur * hbuf + r * Hp + j];
+      const int el = r / n;
+      p.h[((size_t)envs[el].eid * n + (r - el * n)) * H + j] = hs[cur * hbuf + r * Hp + j];
     }
-    if (tid < R) p.last_action[e0 * n + tid] = la[tid];
+    if (tid < R) p.last_action[envs[tid / n].eid * n + tid % n] = la[tid];
     if (tid < ne) {
       const EnvSlot& es = envs[tid];
       if (es.ok) {
-        p.slot[e0 + tid] = es.slot;
-        p.pos[e0 + tid] = es.pos;
-        p.ep_count[e0 + tid] = es.epc;
+        p.slot[es.eid] = es.slot;
+        p.pos[es.eid] = es.pos;
+        p.ep_count[es.eid] = es.epc;
         if (es.pos > 0) p.slot_len[es.slot] = es.pos;
       }
     }

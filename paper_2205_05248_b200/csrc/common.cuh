@@ -64,6 +64,9 @@ struct ActorParams {
   int32_t trace_cap;
   unsigned long long* counters;
   uint32_t* status;
+  // partial step (FFMA kernel only): the call's rows are the M listed environments; null: all E in order
+  const int32_t* env_ids;
+  int32_t M;
 };
 
 // Everything the episode sampler needs (ring_sample.cu).  Passed by value.

@@ -80,7 +80,7 @@ static FfmaWeightOffsets ffma_weight_offsets(int n, int D, int A, int H) {
   return w;
 }
 
-struct StateOffsets { size_t h, last_action, slot, pos, ep_count, counters, status, wff[2], wpack[2], total; };  // two weight images
+struct StateOffsets { size_t h, last_action, slot, pos, ep_count, counters, status, wff[2], wpack[2], ids, total; };  // two weight images
 struct RingOffsets { size_t records, epid, len, complete, total; };
 struct WorkOffsets { size_t obs, avail, reward, done, actions, total; };
 
@@ -114,6 +114,7 @@ static StateOffsets state_offsets(const marl_actor_config_t& c) {
     s.wff[i] = cv.take(ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
     s.wpack[i] = cv.take(tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden));
   }
+  s.ids = cv.take(sizeof(int32_t) * (size_t)c.n_envs);  // environment list of a partial step
   s.total = cv.off;
   return s;
 }
@@ -189,6 +190,7 @@ struct marl_actor {
   cudaEvent_t upload_done, image_free;
   bool image_free_recorded, pending;
   uint64_t pending_version, pending_step;
+  std::vector<uint8_t> id_seen;  // scratch of marl_actor_step_subset
   uint8_t* host_pack2;  // pinned, so that the upload really runs beside the steps
 };
 
@@ -481,10 +483,24 @@ static void fill_params(marl_actor* a, ActorParams& p) {
   p.slot_complete = a->ring + a->ro.complete;
   p.counters = reinterpret_cast<unsigned long long*>(st + a->so.counters);
   p.status = reinterpret_cast<uint32_t*>(st + a->so.status);
+  p.env_ids = nullptr;
+  p.M = c.n_envs;
   p.trace_actions = a->trace_actions;
   p.trace_q = a->trace_q;
   p.trace_first = a->trace_next;
   p.trace_cap = (a->trace_actions || a->trace_q) ? a->trace_cap : 0;
+}
+
+// The published network becomes the one in use: the stream waits for its upload; the image used so far is idle once
+// the work enqueued before this point is done.
+static int switch_to_published(marl_actor* a) {
+  CU_TRY(cudaStreamWaitEvent(a->stream, a->upload_done, 0));
+  CU_TRY(cudaEventRecord(a->image_free, a->stream));
+  a->image_free_recorded = true;
+  a->wslot ^= 1;
+  a->weights_version = a->pending_version;
+  a->pending = false;
+  return MARL_OK;
 }
 
 // Enqueues T steps reading inputs laid out [step][E]...; shared by every stepping entry point.
@@ -507,12 +523,8 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
       done += (size_t)T1 * c.n_envs;
       T -= T1;
     }
-    CU_TRY(cudaStreamWaitEvent(a->stream, a->upload_done, 0));
-    CU_TRY(cudaEventRecord(a->image_free, a->stream));  // the image in use so far is idle once the work above is done
-    a->image_free_recorded = true;
-    a->wslot ^= 1;
-    a->weights_version = a->pending_version;
-    a->pending = false;
+    const int rcs = switch_to_published(a);
+    if (rcs) return rcs;
   }
   ActorParams p;
   fill_params(a, p);
@@ -555,6 +567,53 @@ int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, con
   if (!obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
   if (!(eps >= 0.0f && eps <= 1.0f)) return fail(MARL_EINVAL, "eps must be in [0, 1]");
   return enqueue_steps(a, obs, avail, reward, done, 1, true, eps, 0, 0, 0, actions_out);
+}
+
+int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
+                           const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
+                           int32_t* actions_out) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!env_ids || !obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
+  if (!(eps >= 0.0f && eps <= 1.0f)) return fail(MARL_EINVAL, "eps must be in [0, 1]");
+  const marl_actor_config_t& c = a->cfg;
+  if (M < 1 || M > c.n_envs) return fail(MARL_EINVAL, "M=%d must be in [1, n_envs=%d]", M, c.n_envs);
+  if (!a->have_weights) return fail(MARL_EINVAL, "marl_actor_set_weights has not been called");
+  if (a->step + 1 > 0xFFFFFFFFull) return fail(MARL_EINVAL, "step counter would exceed 32 bits");
+  // every listed environment exists and is listed once: two rows of one environment would race on its state
+  a->id_seen.assign((size_t)c.n_envs, 0);
+  for (int32_t x = 0; x < M; ++x) {
+    const int32_t e = env_ids[x];
+    if (e < 0 || e >= c.n_envs) return fail(MARL_EINVAL, "env_ids[%d]=%d is outside [0, %d)", x, e, c.n_envs);
+    if (a->id_seen[e]) return fail(MARL_EINVAL, "env_ids[%d]=%d is listed twice", x, e);
+    a->id_seen[e] = 1;
+  }
+  if (a->pending && a->step >= a->pending_step) {  // a published network is due
+    const int rcs = switch_to_published(a);
+    if (rcs) return rcs;
+  }
+  int32_t* d_ids = reinterpret_cast<int32_t*>(a->state + a->so.ids);
+  // pageable source: the copy has left the caller's array when the call returns
+  CU_TRY(cudaMemcpyAsync(d_ids, env_ids, sizeof(int32_t) * (size_t)M, cudaMemcpyHostToDevice, a->stream));
+  ActorParams p;
+  fill_params(a, p);
+  p.T = 1;
+  p.t0 = (uint32_t)a->step;
+  p.eps_const_mode = 1;
+  p.eps_const = eps;
+  p.eps_start = p.eps_end = 0;
+  p.anneal_steps = 0;
+  p.obs = obs; p.avail = avail; p.reward = reward; p.done = done;
+  p.obs_step_stride = p.avail_step_stride = p.env_step_stride = 0;
+  p.actions_out = actions_out;
+  p.env_ids = d_ids;
+  p.M = M;
+  ffma_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
+  const int rc = launch_actor_ffma(p, a->sms, a->stream);
+  if (rc < 0) return fail(MARL_ECUDA, "actor kernel launch: %s", cudaGetErrorString((cudaError_t)(-rc)));
+  a->launches += (uint64_t)rc;
+  a->step += 1;
+  if (a->trace_actions || a->trace_q) a->trace_next = a->trace_next + 1 > a->trace_cap ? a->trace_cap : a->trace_next + 1;
+  return MARL_OK;
 }
 
 int marl_actor_step_host(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,

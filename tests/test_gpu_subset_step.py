@@ -1,0 +1,121 @@
+"""The step over a list of environments (asynchronous actors, Sec. III-A): the CUDA library against the oracle,
+call by call, on seeded environment lists of changing size and order."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2205_05248_b200 import binding, workloads
+from referee import NEAR_TIE_BUDGET, RTOL, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _env_block(cfg, T):
+    E = cfg["E"]
+    obs = np.zeros((T, E, cfg["n"], cfg["D"]), np.float32)
+    avail = np.zeros((T, E, cfg["n"], cfg["A"]), np.uint8)
+    rew = np.zeros((T, E), np.float32)
+    done = np.zeros((T, E), np.uint8)
+    for t in range(T):
+        for e in range(E):
+            obs[t, e], avail[t, e], rew[t, e], done[t, e] = oracle.env_emit(cfg, cfg["env"], t, e)
+    return obs, avail, rew, done
+
+
+@pytest.mark.parametrize("prec,shape,full_every", [("fp32", dict(E=96, n=4, A=7, D=24, C=192), 0),
+                                                   ("bf16", dict(E=96, n=4, A=8, D=24, C=192), 5),
+                                                   ("bf16", dict(E=700, n=5, A=11, D=13, C=700), 0),
+                                                   ("fp32", dict(E=3, n=3, A=9, D=30, C=6), 4)])
+def test_subset_steps_match_the_oracle(prec, shape, full_every):
+    cfg = workloads.small_config(H=64, L=5, T=22, precision=prec, env=dict(done_thresh24=1 << 21), **shape)
+    E, n, A, T = cfg["E"], cfg["n"], cfg["A"], cfg["T"]
+    w = workloads.make_weights(cfg)
+    obs, avail, rew, done = _env_block(cfg, T)
+    dev = "cuda:0"
+    d_obs, d_avail, d_rew, d_done = (torch.as_tensor(x, device=dev) for x in (obs, avail, rew, done))
+    actor = binding.Actor(cfg, device=dev)
+    actor.set_weights(w)
+    g_acts, g_q = actor.set_trace(T, want_q=True)
+    sess = oracle.Session(cfg, w, np.arange(E))
+    rng = np.random.default_rng(7)
+    eps, rtol = 0.15, RTOL[prec]
+    near = greedy = 0
+    for t in range(T):
+        if full_every and t % full_every == full_every - 1:
+            ids = np.arange(E)
+            act = actor.step(d_obs[t], d_avail[t], d_rew[t], d_done[t], eps)
+        else:
+            M = int(rng.integers(1, E + 1)) if t % 3 else E          # every third call lists everybody, shuffled
+            ids = rng.permutation(E)[:M].astype(np.int32)
+            tid = torch.as_tensor(ids, device=dev, dtype=torch.long)
+            act = actor.step_subset(ids, d_obs[t].index_select(0, tid).contiguous(),
+                                    d_avail[t].index_select(0, tid).contiguous(), d_rew[t].index_select(0, tid).contiguous(),
+                                    d_done[t].index_select(0, tid).contiguous(), eps)
+        act = act.cpu().numpy()
+        tid = torch.as_tensor(ids, device=dev, dtype=torch.long)
+        q_rows = g_q[t].index_select(0, tid).cpu().numpy()
+        assert np.array_equal(g_acts[t].index_select(0, tid).cpu().numpy(), act)
+        o_act, tr = sess.step_subset(ids, obs[t, ids], avail[t, ids], rew[t, ids], done[t, ids], eps, adopt=act,
+                                     trace=("q", "action_free", "explore"))
+        # the decision follows from the library's own Q row, the mask and the draw keyed by the environment's index
+        N = len(ids) * n
+        re_act, re_ex = oracle.select_batch(q_rows.reshape(N, A), avail[t, ids].reshape(N, A), np.float32(eps),
+                                            cfg["seed"], np.uint32(t), np.repeat(ids.astype(np.uint32), n),
+                                            np.tile(np.arange(n, dtype=np.uint32), len(ids)))
+        assert np.array_equal(re_act, act.reshape(N)), f"call {t}"
+        assert np.array_equal(re_ex, tr["explore"].reshape(N))
+        assert row_rel_err(q_rows, tr["q"]).max() <= rtol, f"call {t}"
+        diff = np.argwhere(tr["action_free"] != act)
+        for (x, i) in diff:
+            gap = abs(float(tr["q"][x, i, tr["action_free"][x, i]]) - float(tr["q"][x, i, act[x, i]]))
+            assert gap <= 1e-4 + 2 * rtol * max(float(np.abs(tr["q"][x, i]).max()), 1e-3)
+        near += len(diff)
+        greedy += int((tr["explore"] == 0).sum())
+        # rows of the trace that were not listed keep the trace's fill value
+        if len(ids) < E:
+            rest = torch.as_tensor(np.setdiff1d(np.arange(E), ids), device=dev, dtype=torch.long)
+            assert bool((g_acts[t].index_select(0, rest) == -7).all())
+    assert near <= max(1, NEAR_TIE_BUDGET[prec] * greedy * 4)
+    torch.cuda.synchronize()
+    st = actor.get_state()
+    for k in ("last_action", "slot", "pos", "ep_count"):
+        assert np.array_equal(st[k].cpu().numpy(), getattr(sess, k)), k
+    assert row_rel_err(st["h"].cpu().numpy(), sess.h).max() <= rtol
+    assert st["step"] == T
+    rv = actor.ring_view()
+    for k in ("slot_epid", "slot_len", "slot_complete"):
+        assert np.array_equal(rv[k].cpu().numpy(), sess.ring[k]), k
+    written = np.arange(cfg["L"])[None, :] < sess.ring["slot_len"][:, None]
+    assert written.sum() > 0
+    for k in ("obs", "avail", "action", "reward", "done"):
+        assert np.array_equal(rv[k].cpu().numpy()[written], sess.ring[k][written]), k
+    assert row_rel_err(rv["q"].cpu().numpy()[written], sess.ring["q"][written]).max() <= rtol
+    status, counters = actor.status()
+    assert status == 0
+    oc = sess.counters
+    assert counters["agent_steps"] == oc[oracle.CNT_STEPS] and counters["episodes"] == oc[oracle.CNT_EPISODES]
+    assert counters["explored"] == oc[oracle.CNT_EXPLORE] and counters["truncated"] == oc[oracle.CNT_TRUNCATED]
+    assert counters["episodes"] > 0
+    actor.destroy()
+
+
+def test_subset_list_is_validated_on_the_host():
+    cfg = workloads.small_config(H=64, D=8, E=16, C=32, L=4, T=4, precision="fp32", n=2, A=4)
+    actor = binding.Actor(cfg)
+    actor.set_weights(workloads.make_weights(cfg))
+    z = lambda *s, dt=torch.float32: torch.zeros(s, dtype=dt, device="cuda:0")
+    def call(ids):
+        M = len(ids)
+        return actor.step_subset(np.array(ids, np.int32), z(M, 2, 8), torch.ones((M, 2, 4), dtype=torch.uint8, device="cuda:0"),
+                                 z(M), z(M, dt=torch.uint8), 0.0)
+    launches = actor.launch_count
+    for bad in ([3, 3], [0, 16], [-1], list(range(16)) + [0]):
+        with pytest.raises(binding.MarlError):
+            call(bad)
+    assert actor.get_state()["step"] == 0 and actor.launch_count == launches
+    call([5, 2])
+    assert actor.get_state()["step"] == 1
+    st = actor.get_state()
+    assert sorted(torch.nonzero(st["pos"]).flatten().tolist()) == [2, 5]
+    actor.destroy()

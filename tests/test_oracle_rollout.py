@@ -199,3 +199,34 @@ def test_weight_switch_uses_the_new_network_from_the_next_step():
     plain, _ = _session(cfg)
     t0 = _roll(plain, cfg, T=4)
     assert all(np.array_equal(t0[k], t1[k]) for k in t0)
+
+
+def test_subset_steps_touch_only_the_listed_environments_and_compose_to_a_full_step():
+    """Asynchronous actors (Sec. III-A): a step over a list of environments is the full step restricted to them.
+    Environments are independent, so stepping two disjoint halves under one step index equals one full step, and
+    an environment that is not listed keeps its state and its part of the pool."""
+    cfg = workloads.small_config(E=6, C=12, L=4, T=10, env=dict(done_thresh24=1 << 22))
+    full, _ = _session(cfg)
+    part, _ = _session(cfg)
+    idle, _ = _session(cfg)
+    a_ids, b_ids = np.array([4, 0, 3]), np.array([1, 5, 2])
+    for t in range(cfg["T"]):
+        outs = [oracle.env_emit(cfg, cfg["env"], t, e) for e in range(cfg["E"])]
+        obs, avail, rew, done = (np.stack([o[k] for o in outs]) for k in range(4))
+        acts, _ = full.step(obs, avail, rew, done, 0.2)
+        before = (idle.h.copy(), idle.pos.copy(), {k: v.copy() for k, v in idle.ring.items()})
+        acts_a, _ = part.step_subset(a_ids, obs[a_ids], avail[a_ids], rew[a_ids], done[a_ids], 0.2)
+        part.t -= 1                                      # the second half belongs to the same step index
+        acts_b, _ = part.step_subset(b_ids, obs[b_ids], avail[b_ids], rew[b_ids], done[b_ids], 0.2)
+        assert np.array_equal(acts[a_ids], acts_a) and np.array_equal(acts[b_ids], acts_b)
+        idle.step_subset(a_ids, obs[a_ids], avail[a_ids], rew[a_ids], done[a_ids], 0.2)
+        S = idle.S
+        for e in b_ids:                                  # not listed: nothing moved
+            assert np.array_equal(idle.h[e], before[0][e]) and idle.pos[e] == before[1][e] == 0
+            for k, v in idle.ring.items():
+                assert np.array_equal(v[e * S:(e + 1) * S], before[2][k][e * S:(e + 1) * S]), k
+    for k in ("h", "last_action", "slot", "pos", "ep_count"):
+        assert np.array_equal(getattr(full, k), getattr(part, k)), k
+    for k in full.ring:
+        assert np.array_equal(full.ring[k], part.ring[k]), k
+    assert np.array_equal(full.counters, part.counters)
