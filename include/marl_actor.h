@@ -211,8 +211,8 @@ int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, con
  * over the list: row x belongs to environment env_ids[x]: obs f32[M][n][D], avail u8[M][n][A], reward f32[M],
  * done u8[M], actions_out i32[M][n] (may be NULL).  The call consumes one index of the global step counter, which
  * keys the exploration stream as (seed, step, environment, agent) with the environment's own index; a trace row
- * of this step is written at the environment's own index as well.  Runs on the CUDA-core kernel for every shape
- * and precision. */
+ * of this step is written at the environment's own index as well.  Runs on the pipelined tensor-core kernel where
+ * the actor uses it and the arrays can be bulk-copied (16-byte aligned obs and avail), else on the CUDA-core kernel. */
 int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
                            const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
                            int32_t* actions_out);

@@ -30,6 +30,7 @@
 // hand-offs are mbarriers with bounded waits; an expired wait sets MARL_STATUS_TIMEOUT and lets the block run
 // to its end with every index in range.
 #include <cstring>
+#include <type_traits>
 
 #include "actor_tc_layout.cuh"
 #include "common.cuh"
@@ -197,7 +198,10 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
   __syncwarp();
 }
 
-template <int NQ, bool PLAIN>  // PLAIN: the word-by-word path of shapes whose per-environment blocks are not 16-byte multiples
+// PLAIN: the word-by-word path of shapes whose per-environment blocks are not 16-byte multiples.
+// LIST: the call's rows are the environments of p.env_ids (a partial step); inputs, the last step's actions and the
+// tiling follow the row, state, ring cursors, the draw's key and the trace follow the environment.
+template <int NQ, bool PLAIN, bool LIST>
 __global__ void __launch_bounds__(TP_THREADS, 1)
     actor_tcp_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TpLayout L) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -370,17 +374,18 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
       uint32_t done_next = 0;
       uint32_t q = 0, qslot = 0, qpar = 1, kstep = 0;  // chunk index, q % NS, parity of the slot's previous use, global step
       for (; tile < p.num_tiles; tile += gridDim.x) {
-        const int ne = min(L.ept, p.E - tile * L.ept);
+        const int ne = min(L.ept, p.M - tile * L.ept);
         const int nck = (ne + TP_G - 1) / TP_G;
-        const int e = tile * L.ept + lane;
+        const int x = tile * L.ept + lane;  // row of the call
         const bool mine = lane < ne;
+        const int e = (LIST && mine) ? __ldg(p.env_ids + x) : x;
         ok = 0;
         if (mine) {
           slot = p.slot[e];
           pos = p.pos[e];
           epc = p.ep_count[e];
           ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
-          done_next = p.done[e];
+          done_next = p.done[x];
         }
         for (int s = 0; s < T; ++s, ++kstep) {
           unsigned long long rec = 0;
@@ -399,7 +404,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           dstp_s[(kstep & (TP_DST_DEPTH - 1)) * 32 + lane] = rec;
           closes = __any_sync(0xFFFFFFFFu, closes);
           if (lane == 0) closeany_s[kstep & (TP_DST_DEPTH - 1)] = closes;
-          if (mine && s + 1 < T) done_next = p.done[(size_t)(s + 1) * p.env_step_stride + e];
+          if (mine && s + 1 < T) done_next = p.done[(size_t)(s + 1) * p.env_step_stride + x];
           __syncwarp();
           for (int c = 0; c < nck; ++c) {
             const int ge = min(TP_G, ne - c * TP_G);
@@ -430,9 +435,10 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
       unsigned long long c_episodes = 0, c_trunc = 0;
       uint32_t st_bits = 0, sd = 0, it = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        const int ne = min(L.ept, p.E - tile * L.ept);
+        const int ne = min(L.ept, p.M - tile * L.ept);
         const bool mine = lane < ne;
-        const int e = tile * L.ept + lane;
+        const int x = tile * L.ept + lane;  // row of the call
+        const int e = (LIST && mine) ? __ldg(p.env_ids + x) : x;
         int32_t slot = 0, pos = 0, ok = 0;
         long long epc = 0;
         float reward_next = 0.f;
@@ -443,8 +449,8 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           epc = p.ep_count[e];
           ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
           if (!ok) st_bits |= MARL_STATUS_BAD_INDEX;
-          reward_next = p.reward[e];
-          done_next = p.done[e];
+          reward_next = p.reward[x];
+          done_next = p.done[x];
         }
         // Copies the tails of one step (buffer bb, record addresses in tdst_s) to the ring: 16 bytes per lane, the
         // pieces of all environments in one flat loop.
@@ -482,8 +488,8 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           TP_STAMP(lane == 0, it, 21);
           if (s > 0) copy_tails(b ^ 1u);           // then the previous step's tails, off the critical path
           if (mine && s + 1 < T) {
-            reward_next = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
-            done_next = p.done[(size_t)(s + 1) * p.env_step_stride + e];
+            reward_next = p.reward[(size_t)(s + 1) * p.env_step_stride + x];
+            done_next = p.done[(size_t)(s + 1) * p.env_step_stride + x];
           }
           mbar_wait(&B->stepd, sd & 1, abortf);  // action and Q of step s are in the tail
           TP_STAMP(lane == 0, it, 20);
@@ -519,7 +525,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
       // issued as soon as the chunk has arrived; a slot is handed back once its stores have been read out.
       uint32_t q = 0, qslot = 0, qpar = 0, pslot = 0, kstep = 0;
       for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        const int ne = min(L.ept, p.E - tile * L.ept);
+        const int ne = min(L.ept, p.M - tile * L.ept);
         const int nck = (ne + TP_G - 1) / TP_G;
         for (int s = 0; s < T; ++s, ++kstep) {
           for (int c = 0; c < nck; ++c) {
@@ -562,7 +568,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
     uint32_t it = 0, qbase = 0;  // steps and chunks before this step
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
-      const int ne = min(L.ept, p.E - e0);
+      const int ne = min(L.ept, p.M - e0);
       const int nck = (ne + TP_G - 1) / TP_G;
       for (int s = 0; s < T; ++s) {
         const uint32_t t = p.t0 + (uint32_t)s;
@@ -670,7 +676,8 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const int rel = ci / n, rai = ci - rel * n;
           const uint32_t mask = sel[ci].x;
           int pick = -1;
-          if (mask != 0) pick = draw_explore(mask, eps, p.seed, t, (uint32_t)(e0 + rel), (uint32_t)rai);
+          if (mask != 0)
+            pick = draw_explore(mask, eps, p.seed, t, (uint32_t)(LIST ? __ldg(p.env_ids + e0 + rel) : e0 + rel), (uint32_t)rai);
           sel[ci].y = (uint32_t)pick;
         }
         warp_arrive(&B->selready[it & 3], lane);
@@ -691,11 +698,11 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
-      const int ne = min(L.ept, p.E - e0);
+      const int ne = min(L.ept, p.M - e0);
       const int R = ne * n;
       const bool live = row < R;
       const bool is_row = live && half == 0;  // owner of the row's choice
-      const int e = e0 + el;
+      const int e = (LIST && live) ? __ldg(p.env_ids + e0 + el) : e0 + el;
       const size_t grow = (size_t)e * n + ai;  // global row
       int la = -1;
 
@@ -881,7 +888,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
                   if (a < A) p.trace_q[trow * A + a] = __uint_as_float(qv[a]);
               }
             }
-            if (p.actions_out && s == T - 1) p.actions_out[grow] = act;
+            if (p.actions_out && s == T - 1) p.actions_out[LIST ? (size_t)(e0 + el) * n + ai : grow] = act;
           }
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -932,14 +939,19 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
   const TpLayout L = tp_layout(p_in.n, p_in.D, p_in.A, (int)p_in.rl.rec_bytes);
   ActorParams p = p_in;
   p.ept = L.ept;  // (tiles of whole chunks for the plain shapes)
-  p.num_tiles = (p.E + L.ept - 1) / L.ept;
+  p.num_tiles = (p.M + L.ept - 1) / L.ept;
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
-  if (L.plain && p.E % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
-  auto kernel = L.NQ == 16 ? (L.plain ? actor_tcp_kernel<16, true> : actor_tcp_kernel<16, false>)
-                           : (L.plain ? actor_tcp_kernel<32, true> : actor_tcp_kernel<32, false>);
-  static uint32_t configured[4] = {0, 0, 0, 0};
-  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0)];
+  if (L.plain && p.M % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
+  const bool list = p.env_ids != nullptr;
+  auto pick = [&](auto nq) {
+    constexpr int Q = decltype(nq)::value;
+    return list ? (L.plain ? actor_tcp_kernel<Q, true, true> : actor_tcp_kernel<Q, false, true>)
+                : (L.plain ? actor_tcp_kernel<Q, true, false> : actor_tcp_kernel<Q, false, false>);
+  };
+  auto kernel = L.NQ == 16 ? pick(std::integral_constant<int, 16>()) : pick(std::integral_constant<int, 32>());
+  static uint32_t configured[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + (list ? 4 : 0)];
   if (L.total > conf) {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return -(int)e;

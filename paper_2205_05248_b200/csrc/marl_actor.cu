@@ -607,8 +607,15 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
   p.actions_out = actions_out;
   p.env_ids = d_ids;
   p.M = M;
-  ffma_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
-  const int rc = launch_actor_ffma(p, a->sms, a->stream);
+  int rc = 0;
+  if (a->use_tcp) {  // 0: these pointers or this list length cannot be bulk-copied
+    tc_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
+    rc = launch_actor_tcp(p, a->sms, a->stream);
+  }
+  if (rc == 0) {
+    ffma_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
+    rc = launch_actor_ffma(p, a->sms, a->stream);
+  }
   if (rc < 0) return fail(MARL_ECUDA, "actor kernel launch: %s", cudaGetErrorString((cudaError_t)(-rc)));
   a->launches += (uint64_t)rc;
   a->step += 1;

@@ -23,19 +23,25 @@ def _env_block(cfg, T):
     return obs, avail, rew, done
 
 
-@pytest.mark.parametrize("prec,shape,full_every", [("fp32", dict(E=96, n=4, A=7, D=24, C=192), 0),
-                                                   ("bf16", dict(E=96, n=4, A=8, D=24, C=192), 5),
-                                                   ("bf16", dict(E=700, n=5, A=11, D=13, C=700), 0),
-                                                   ("fp32", dict(E=3, n=3, A=9, D=30, C=6), 4)])
-def test_subset_steps_match_the_oracle(prec, shape, full_every):
+@pytest.mark.parametrize("prec,kernel,shape,full_every", [
+    ("fp32", "ffma", dict(E=96, n=4, A=7, D=24, C=192), 0),
+    ("bf16", "ffma", dict(E=700, n=5, A=11, D=13, C=700), 0),
+    ("fp32", "ffma", dict(E=3, n=3, A=9, D=30, C=6), 4),
+    # the pipelined tensor-core kernel: bulk-copied rows; several tiles with a ragged last one and partial chunks
+    ("bf16", "pipelined", dict(E=96, n=4, A=8, D=24, C=192), 5),
+    ("bf16", "pipelined", dict(E=700, n=8, A=14, D=80, C=700), 0),
+    # rows that are not 16-byte multiples: lists whose length is not a multiple of four go to the CUDA-core kernel
+    ("bf16", "pipelined", dict(E=300, n=5, A=12, D=55, C=300), 6)])
+def test_subset_steps_match_the_oracle(prec, kernel, shape, full_every):
     cfg = workloads.small_config(H=64, L=5, T=22, precision=prec, env=dict(done_thresh24=1 << 21), **shape)
     E, n, A, T = cfg["E"], cfg["n"], cfg["A"], cfg["T"]
     w = workloads.make_weights(cfg)
     obs, avail, rew, done = _env_block(cfg, T)
     dev = "cuda:0"
     d_obs, d_avail, d_rew, d_done = (torch.as_tensor(x, device=dev) for x in (obs, avail, rew, done))
-    actor = binding.Actor(cfg, device=dev)
+    actor = binding.Actor(cfg, device=dev, kernel=kernel)
     actor.set_weights(w)
+    assert actor.kernel_name == {"ffma": "ffma", "pipelined": "tcgen05-pipelined"}[kernel]
     g_acts, g_q = actor.set_trace(T, want_q=True)
     sess = oracle.Session(cfg, w, np.arange(E))
     rng = np.random.default_rng(7)
