@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--refresh", action="store_true",
                     help="publish a new network during every step, effective at the middle of the next rollout "
                          "(the learner's model update running beside the workers)")
+    ap.add_argument("--subset", type=float, default=0.0, metavar="FRACTION",
+                    help="time marl_actor_step_subset instead: every call steps a seeded list of FRACTION * E "
+                         "environments (a multiple of four), T calls per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sampler", type=int, default=0, metavar="B",
@@ -279,6 +282,66 @@ def run_sampler(args, cfg, dev):
     actor.destroy()
 
 
+def run_subset(args, cfg, dev):
+    """--subset FRACTION: T calls of marl_actor_step_subset per step, each over one of four seeded lists of
+    M = FRACTION * E environments in random order, the dense inputs of each list resident in HBM beforehand.
+    Algorithmic bytes per agent-step: the one-step figure (hidden state loaded and stored by every call) plus the
+    list entry."""
+    import numpy as np
+    import torch
+    from paper_2205_05248_b200 import binding, workloads
+    T, E, n = cfg["T"], cfg["E"], cfg["n"]
+    M = max(4, int(args.subset * E) // 4 * 4)
+    weights = workloads.make_weights(cfg)
+    actor = binding.Actor(cfg, device=str(dev), kernel=args.kernel, work_steps=1)
+    actor.set_weights(weights)
+    staged = actor.env_generate(cfg["env"], 0, 4)
+    rng = np.random.default_rng(cfg["seed"])
+    lists = [rng.permutation(E)[:M].astype(np.int32) for _ in range(4)]
+    inputs = []
+    for k, ids in enumerate(lists):
+        tid = torch.as_tensor(ids, device=dev, dtype=torch.long)
+        inputs.append([t[k].index_select(0, tid).contiguous() for t in staged])
+    acts = torch.empty((M, n), dtype=torch.int32, device=dev)
+    del staged
+
+    def one_step():
+        for k in range(T):
+            actor.step_subset(lists[k % 4], *inputs[k % 4], cfg["eps_start"], acts)
+
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize()
+    launches0 = actor.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        one_step()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    launches = actor.launch_count - launches0
+    status, _ = actor.status()
+    assert status == 0, f"device status {status}"
+    per_step = algorithmic_bytes_per_agent_step(cfg, 1) + 4.0 / n
+    kernel_ms = ms / launches
+    achieved = per_step * M * n / (kernel_ms * 1e-3) / 1e9
+    peaks, peak_kind = load_peaks()
+    in_bytes = sum(t.numel() * t.element_size() for t in inputs[0])
+    print(json.dumps({"metric": METRIC, "value": M * n * T * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+                      "higher_is_better": True, "dtype": cfg["precision"], "data": "synthetic",
+                      "config": {"workload": cfg["name"], "E": E, "M": M, "n": n, "T": T, "kernel": actor.kernel_name,
+                                 "step": f"T={T} marl_actor_step_subset calls over lists of M={M} of E={E} environments",
+                                 "l2": f"each call reads {in_bytes / 1e6:.0f} MB of inputs and {M * n * cfg['H'] * 4 / 1e6:.0f} MB of "
+                                       "hidden state (four lists in turn)"},
+                      "gpu_launches": int(launches),
+                      "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
+                                   "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": per_step}}), flush=True)
+    actor.destroy()
+
+
 def main():
     args = parse_args()
     from paper_2205_05248_b200 import workloads
@@ -298,6 +361,10 @@ def main():
     if args.sampler > 0:
         if rank == 0:
             run_sampler(args, cfg, dev)
+        return
+    if args.subset > 0:
+        if rank == 0:
+            run_subset(args, cfg, dev)
         return
     cfg["seed"] = cfg["seed"] + (rank << 20)          # every rank runs its own replica
     cfg["env"] = dict(cfg["env"], seed=cfg["env"]["seed"] + (rank << 20))
