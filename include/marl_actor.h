@@ -217,6 +217,18 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
                            const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
                            int32_t* actions_out);
 
+/* marl_actor_step_subset for environments that answer after the action (Algorithm 1: put o, get a, then
+ * "o, r <- Env.step(a)"): prev_reward f32[M] and prev_done u8[M] (device) are the outcome of each listed
+ * environment's PREVIOUS action and arrive with this observation.  Per environment, in this order: if a record of
+ * the open episode waits for its outcome (cursor > 0), the outcome is written into it and, if the game ended or
+ * the slot is full, the episode is closed (header, counters, next slot, zero hidden state, no last action); then
+ * the decision on this observation is recorded with reward 0 and done 0 for now.  An environment's first call has
+ * nothing waiting: its prev_reward / prev_done are ignored.  Do not mix with the synchronous stepping calls on one
+ * actor (they close an episode in the step that ends it).  Runs on the CUDA-core kernel. */
+int marl_actor_step_lagged(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
+                           const uint8_t* avail, const float* prev_reward, const uint8_t* prev_done, float eps,
+                           int32_t* actions_out);
+
 /* The same step with HOST buffers (the observation-action pipe of Algorithms 1 and 2 when the simulators
  * run on the host): copies the four inputs to the device, runs the step, copies the actions back and
  * SYNCHRONISES the stream before returning.  Pinned host memory makes the copies asynchronous. */

@@ -307,7 +307,13 @@ class Session:
         self.t += 1
         return actions, {k: v[0] for k, v in tr.items() if v is not None}
 
-    def step_subset(self, env_ids, obs, avail, reward, done, eps: float, adopt=None, trace=()):
+    def step_lagged(self, env_ids, obs, avail, prev_reward, prev_done, eps: float, adopt=None, trace=()):
+        """step_subset when the environment answers after the action (Algorithm 1: the reward of an action comes
+        back with the next observation): prev_reward / prev_done belong to each environment's previous action."""
+        return self.step_subset(env_ids, obs, avail, prev_reward, prev_done, eps, adopt=adopt, trace=trace,
+                                lagged=True)
+
+    def step_subset(self, env_ids, obs, avail, reward, done, eps: float, adopt=None, trace=(), lagged=False):
         """One decision step for the listed environments only (actors are asynchronous, Sec. III-A: the worker
         serves the observations that have arrived).  Index plumbing around the same step routine: the listed rows of
         the state and of the pool image are copied out, stepped with the session's step counter, and copied back;
@@ -335,10 +341,16 @@ class Session:
             rg = _Ring(*[_ptr(rsub[k]) for k in names])
         tr, ts = self._alloc_trace(1, set(trace or ()), rows=M)
         actions = np.zeros((M, n), np.int32)
-        lib().oracle_step(C.byref(self._d), C.byref(self._w), _ptr(ids), C.c_int32(M), C.c_uint32(self.t),
-                          C.c_float(eps), _ptr(obs), _ptr(avail), _ptr(reward), _ptr(done), _ptr(adopt), C.byref(st),
-                          C.byref(rg) if rg is not None else None, _ptr(actions), C.byref(ts), C.c_int32(0),
-                          _ptr(self.counters), C.c_int32(self.n_threads))
+        if lagged:
+            lib().oracle_step_lagged(C.byref(self._d), C.byref(self._w), _ptr(ids), C.c_int32(M), C.c_uint32(self.t),
+                                     C.c_float(eps), _ptr(obs), _ptr(avail), _ptr(reward), _ptr(done), _ptr(adopt),
+                                     C.byref(st), C.byref(rg) if rg is not None else None, _ptr(actions), C.byref(ts),
+                                     _ptr(self.counters))
+        else:
+            lib().oracle_step(C.byref(self._d), C.byref(self._w), _ptr(ids), C.c_int32(M), C.c_uint32(self.t),
+                              C.c_float(eps), _ptr(obs), _ptr(avail), _ptr(reward), _ptr(done), _ptr(adopt),
+                              C.byref(st), C.byref(rg) if rg is not None else None, _ptr(actions), C.byref(ts),
+                              C.c_int32(0), _ptr(self.counters), C.c_int32(self.n_threads))
         for k, v in sub.items():
             getattr(self, k)[loc] = v
         if rsub is not None:

@@ -524,6 +524,97 @@ void oracle_step(const oracle_dims* d, const oracle_weights* w, const int32_t* e
 }
 
 // ---------------------------------------------------------------------------------------------------
+// The same step when the environment answers after the action (Algorithm 1: put o, get a, then
+// "o, r <- Env.step(a)"): the reward and the end-of-game flag of an action reach the worker with the NEXT
+// observation of that environment.  For each listed environment, in this order:
+//   1. if a record of the open episode is still waiting for its outcome (pos > 0): prev_reward / prev_done
+//      are written into that record (pos - 1); if the game ended, or the slot is full (pos == L), the
+//      episode closes exactly as in the synchronous step (header, counters, next slot, zero hidden state,
+//      no last action);
+//   2. the decision on this observation, recorded at (slot, pos) with reward 0 and done 0 for now;
+//      the cursor moves on and the slot's length counts the new record.
+// An environment's first call has nothing waiting, so its prev_reward / prev_done are ignored.
+// ---------------------------------------------------------------------------------------------------
+void oracle_step_lagged(const oracle_dims* d, const oracle_weights* w, const int32_t* env_ids, int32_t Es,
+                        uint32_t t, float eps, const float* obs, const uint8_t* avail,
+                        const float* prev_reward, const uint8_t* prev_done, const int32_t* adopt,
+                        oracle_state* st, oracle_ring* ring, int32_t* actions_out, oracle_trace* tr,
+                        uint64_t* counters) {
+  const int n = d->n_agents, D = d->obs_dim, A = d->n_actions, H = d->hidden, L = d->ring_steps;
+  const int E = d->n_envs;
+  const int S = d->ring_episodes / E;
+  std::vector<float> q(A), hnew((size_t)n * H);
+  for (int x = 0; x < Es; ++x) {
+    const int e = env_ids[x];
+    // ---- 1. the outcome of the previous action ----
+    if (st->pos[x] > 0) {
+      const int pos = st->pos[x];
+      const size_t rs = (size_t)x * S + (st->slot[x] - e * S);
+      if (ring) {
+        ring->reward[rs * L + pos - 1] = prev_reward[x];
+        ring->done[rs * L + pos - 1] = prev_done[x];
+      }
+      const bool ended = prev_done[x] != 0;
+      if (ended || pos == L) {
+        if (ring) ring->slot_complete[rs] = 1;
+        counters[ORACLE_CNT_EPISODES] += 1;
+        if (!ended) counters[ORACLE_CNT_TRUNCATED] += 1;
+        st->ep_count[x] += 1;
+        st->slot[x] = e * S + (int)(st->ep_count[x] % S);
+        st->pos[x] = 0;
+        for (int k = 0; k < n * H; ++k) st->h[(size_t)x * n * H + k] = 0.0f;
+        for (int i = 0; i < n; ++i) st->last_action[x * n + i] = -1;
+      }
+    }
+    // ---- 2. the decision on this observation ----
+    const int slot = st->slot[x], pos = st->pos[x];
+    const size_t rs = (size_t)x * S + (slot - e * S);
+    if (ring && pos == 0) {
+      ring->slot_epid[rs] = st->ep_count[x] * (int64_t)E + e;
+      ring->slot_len[rs] = 0;
+      ring->slot_complete[rs] = 0;
+    }
+    for (int i = 0; i < n; ++i) {
+      const size_t row = (size_t)x * n + i;
+      const float* o = obs + row * D;
+      const uint8_t* av = avail + row * A;
+      oracle_agent_forward(d, w, o, i, st->last_action[row], st->h + row * H, q.data(),
+                           hnew.data() + (size_t)i * H);
+      uint8_t ex = 0, na = 0;
+      float u = 0.f;
+      const int32_t a_free = oracle_select_action(q.data(), av, A, eps, d->seed, t, (uint32_t)e,
+                                                  (uint32_t)i, &ex, &u, &na);
+      const int32_t a_used = adopt ? adopt[row] : a_free;
+      counters[ORACLE_CNT_STEPS] += 1;
+      counters[ORACLE_CNT_EXPLORE] += ex;
+      counters[ORACLE_CNT_NO_AVAIL] += na;
+      if (actions_out) actions_out[row] = a_used;
+      if (ring) {
+        const size_t rr = (rs * L + pos) * n + i;
+        std::memcpy(ring->obs + rr * D, o, sizeof(float) * D);
+        std::memcpy(ring->avail + rr * A, av, A);
+        std::memcpy(ring->q + rr * A, q.data(), sizeof(float) * A);
+        ring->action[rr] = a_used;
+      }
+      if (tr) {
+        const size_t trow = (size_t)x * n + i;
+        if (tr->q) std::memcpy(tr->q + trow * A, q.data(), sizeof(float) * A);
+        if (tr->action_free) tr->action_free[trow] = a_free;
+        if (tr->explore) tr->explore[trow] = ex;
+      }
+      st->last_action[row] = a_used;
+    }
+    if (ring) {
+      ring->reward[rs * L + pos] = 0.0f;
+      ring->done[rs * L + pos] = 0;
+      ring->slot_len[rs] = pos + 1;
+    }
+    st->pos[x] = pos + 1;
+    std::memcpy(st->h + (size_t)x * n * H, hnew.data(), sizeof(float) * (size_t)n * H);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // T steps against the synthetic environment, starting at global step t0.
 //   adopt [T][Es][n] or null (see oracle_step).  eps follows oracle_eps_at with the global step index.
 // Each thread owns a range of environments and walks its own steps; the result does not depend on

@@ -24,7 +24,7 @@ STATUS_NO_AVAIL, STATUS_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4
 EXPORTS = [
     "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_publish_weights",
     "marl_actor_weights_version",
-    "marl_actor_step", "marl_actor_step_subset", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
+    "marl_actor_step", "marl_actor_step_subset", "marl_actor_step_lagged", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
     "marl_actor_set_trace", "marl_ring_view", "marl_ring_sample", "marl_actor_get_state", "marl_actor_set_state",
     "marl_actor_status", "marl_actor_reset", "marl_actor_destroy", "marl_actor_kernel_name",
     "marl_actor_launch_count", "marl_last_error", "marl_rollout_noalloc", "marl_selftest_bounded_wait",
@@ -107,6 +107,7 @@ def load_library():
         lib.marl_actor_step.argtypes = [P, P, P, P, P, C.c_float, P]
         lib.marl_actor_step_host.argtypes = [P, P, P, P, P, C.c_float, P]
         lib.marl_actor_step_subset.argtypes = [P, P, C.c_int32, P, P, P, P, C.c_float, P]
+        lib.marl_actor_step_lagged.argtypes = [P, P, C.c_int32, P, P, P, P, C.c_float, P]
         lib.marl_env_generate.argtypes = [P, C.POINTER(SynthEnv), C.c_uint32, C.c_int32, P, P, P, P]
         lib.marl_rollout_staged.argtypes = [P, P, P, P, P, C.c_int32, C.c_double, C.c_double, C.c_int32]
         lib.marl_rollout.argtypes = [P, C.POINTER(SynthEnv), C.c_int32, C.c_double, C.c_double, C.c_int32]
@@ -252,7 +253,11 @@ class Actor:
                                         C.c_float(eps), _dptr(actions_out)))
         return actions_out
 
-    def step_subset(self, env_ids, obs, avail, reward, done, eps: float, actions_out=None):
+    def step_lagged(self, env_ids, obs, avail, prev_reward, prev_done, eps: float, actions_out=None):
+        """marl_actor_step_lagged: step_subset with the outcome of each environment's previous action."""
+        return self.step_subset(env_ids, obs, avail, prev_reward, prev_done, eps, actions_out, lagged=True)
+
+    def step_subset(self, env_ids, obs, avail, reward, done, eps: float, actions_out=None, lagged=False):
         """marl_actor_step_subset: env_ids is a host int32 array [M]; the other tensors are device tensors over the
         list.  Returns the int32 [M][n] action tensor."""
         import numpy as np
@@ -262,9 +267,9 @@ class Actor:
             actions_out = torch.empty((M, n), dtype=torch.int32, device=self.device)
         for t, dt in ((obs, torch.float32), (avail, torch.uint8), (reward, torch.float32), (done, torch.uint8)):
             assert t.is_cuda and t.dtype == dt and t.is_contiguous() and t.shape[0] == M
-        _check(self.lib.marl_actor_step_subset(self.handle, ids.ctypes.data_as(C.c_void_p), C.c_int32(M), _dptr(obs),
-                                               _dptr(avail), _dptr(reward), _dptr(done), C.c_float(eps),
-                                               _dptr(actions_out)))
+        fn = self.lib.marl_actor_step_lagged if lagged else self.lib.marl_actor_step_subset
+        _check(fn(self.handle, ids.ctypes.data_as(C.c_void_p), C.c_int32(M), _dptr(obs), _dptr(avail), _dptr(reward),
+                  _dptr(done), C.c_float(eps), _dptr(actions_out)))
         return actions_out
 
     def step_host(self, obs, avail, reward, done, eps: float, actions_out):

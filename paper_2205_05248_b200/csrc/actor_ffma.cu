@@ -161,11 +161,39 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       s.reward = 0.f;
       s.done = 0;
       s.reset = 0;
-      s.ok = (s.slot >= 0 && s.slot < p.E * p.S && s.pos >= 0 && s.pos < p.L) ? 1 : 0;
+      // (with late outcomes a full slot waits, at pos == L, for its last outcome before it is truncated)
+      s.ok = (s.slot >= 0 && s.slot < p.E * p.S && s.pos >= 0 && s.pos < p.L + (p.lagged ? 1 : 0)) ? 1 : 0;
       if (!s.ok) st_bits |= MARL_STATUS_BAD_INDEX;
+      if (p.lagged && s.ok && s.pos > 0) {
+        // The outcome of the previous action arrives with this observation: it completes the record at pos - 1 and,
+        // if the game ended or the slot is full, closes the episode before this step's decision.
+        const float r = p.reward[e0 + tid];
+        const int d = p.done[e0 + tid] ? 1 : 0;
+        uint8_t* rec = p.ring + (size_t)s.slot * p.slot_stride + (size_t)(s.pos - 1) * p.rl.rec_bytes;
+        *reinterpret_cast<float*>(rec + p.rl.off_reward) = r;
+        rec[p.rl.off_done] = (uint8_t)d;
+        if (d || s.pos == p.L) {
+          p.slot_len[s.slot] = s.pos;
+          p.slot_complete[s.slot] = 1;
+          c_episodes += 1;
+          if (!d) c_trunc += 1;
+          s.epc += 1;
+          s.slot = s.eid * p.S + (int)(s.epc % p.S);
+          s.pos = 0;
+          s.reset = 1;
+        }
+      }
       envs[tid] = s;
     }
     __syncthreads();
+    if (p.lagged) {  // an episode closed above starts from a zero hidden state and no last action
+      for (int idx = tid; idx < R * H; idx += FF_THREADS) {
+        const int r = idx / H, j = idx - r * H;
+        if (envs[r / n].reset) hs[r * Hp + j] = 0.f;
+      }
+      if (tid < R && envs[tid / n].reset) la[tid] = -1;
+      __syncthreads();
+    }
 
     for (int s = 0; s < p.T; ++s) {
       const uint32_t t = p.t0 + (uint32_t)s;
@@ -223,8 +251,8 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         }
         if (tid < ne) {
           EnvSlot& es = envs[tid];
-          es.reward = p.reward[(size_t)s * p.env_step_stride + e0 + tid];
-          es.done = p.done[(size_t)s * p.env_step_stride + e0 + tid] ? 1 : 0;
+          es.reward = p.lagged ? 0.f : p.reward[(size_t)s * p.env_step_stride + e0 + tid];
+          es.done = (!p.lagged && p.done[(size_t)s * p.env_step_stride + e0 + tid]) ? 1 : 0;
           es.reset = 0;
           if (es.ok && es.pos == 0) {  // an episode opens in this slot
             p.slot_epid[es.slot] = es.epc * (long long)p.E + es.eid;
@@ -418,7 +446,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           uint8_t* rec = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes;
           *reinterpret_cast<float*>(rec + p.rl.off_reward) = es.reward;
           rec[p.rl.off_done] = (uint8_t)es.done;
-          const bool full = es.pos + 1 == p.L;
+          const bool full = !p.lagged && es.pos + 1 == p.L;  // (late outcomes: the next call truncates)
           if (es.done || full) {
             p.slot_len[es.slot] = es.pos + 1;
             p.slot_complete[es.slot] = 1;

@@ -67,6 +67,8 @@ struct ActorParams {
   // partial step (FFMA kernel only): the call's rows are the M listed environments; null: all E in order
   const int32_t* env_ids;
   int32_t M;
+  // FFMA kernel, T == 1: reward/done are the outcome of each environment's PREVIOUS action (committed at pos - 1)
+  int32_t lagged;
 };
 
 // Everything the episode sampler needs (ring_sample.cu).  Passed by value.

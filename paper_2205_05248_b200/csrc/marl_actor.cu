@@ -485,6 +485,7 @@ static void fill_params(marl_actor* a, ActorParams& p) {
   p.status = reinterpret_cast<uint32_t*>(st + a->so.status);
   p.env_ids = nullptr;
   p.M = c.n_envs;
+  p.lagged = 0;
   p.trace_actions = a->trace_actions;
   p.trace_q = a->trace_q;
   p.trace_first = a->trace_next;
@@ -513,7 +514,7 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   if (a->pending && a->step + (uint64_t)T > a->pending_step) {
     // A published network takes effect inside this span: the steps before it run on the current image, then the
     // stream waits for the upload (which has been running beside the earlier steps) and the images are swapped.
-    const int T1 = (int)(a->pending_step - a->step);
+    const int T1 = a->pending_step > a->step ? (int)(a->pending_step - a->step) : 0;
     if (T1 > 0) {
       const int rc1 = enqueue_steps(a, obs, avail, reward, done, T1, eps_const, eps, eps_start, eps_end, anneal, nullptr);
       if (rc1) return rc1;
@@ -569,9 +570,11 @@ int marl_actor_step(marl_actor_t* a, const float* obs, const uint8_t* avail, con
   return enqueue_steps(a, obs, avail, reward, done, 1, true, eps, 0, 0, 0, actions_out);
 }
 
-int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
-                           const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
-                           int32_t* actions_out) {
+}  // extern "C"
+
+// One step over a host list of environments; lagged: reward/done belong to each environment's previous action.
+static int step_list(marl_actor* a, const int32_t* env_ids, int32_t M, const float* obs, const uint8_t* avail,
+                     const float* reward, const uint8_t* done, float eps, int32_t* actions_out, bool lagged) {
   if (!a) return fail(MARL_EINVAL, "actor is NULL");
   if (!env_ids || !obs || !avail || !reward || !done) return fail(MARL_EINVAL, "an input pointer is NULL");
   if (!(eps >= 0.0f && eps <= 1.0f)) return fail(MARL_EINVAL, "eps must be in [0, 1]");
@@ -607,8 +610,9 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
   p.actions_out = actions_out;
   p.env_ids = d_ids;
   p.M = M;
+  p.lagged = lagged ? 1 : 0;
   int rc = 0;
-  if (a->use_tcp) {  // 0: these pointers or this list length cannot be bulk-copied
+  if (a->use_tcp && !lagged) {  // 0: these pointers or this list length cannot be bulk-copied
     tc_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
     rc = launch_actor_tcp(p, a->sms, a->stream);
   }
@@ -621,6 +625,20 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
   a->step += 1;
   if (a->trace_actions || a->trace_q) a->trace_next = a->trace_next + 1 > a->trace_cap ? a->trace_cap : a->trace_next + 1;
   return MARL_OK;
+}
+
+extern "C" {
+
+int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
+                           const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
+                           int32_t* actions_out) {
+  return step_list(a, env_ids, M, obs, avail, reward, done, eps, actions_out, false);
+}
+
+int marl_actor_step_lagged(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
+                           const uint8_t* avail, const float* prev_reward, const uint8_t* prev_done, float eps,
+                           int32_t* actions_out) {
+  return step_list(a, env_ids, M, obs, avail, prev_reward, prev_done, eps, actions_out, true);
 }
 
 int marl_actor_step_host(marl_actor_t* a, const float* obs, const uint8_t* avail, const float* reward,

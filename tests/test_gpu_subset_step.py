@@ -125,3 +125,68 @@ def test_subset_list_is_validated_on_the_host():
     st = actor.get_state()
     assert sorted(torch.nonzero(st["pos"]).flatten().tolist()) == [2, 5]
     actor.destroy()
+
+
+@pytest.mark.parametrize("prec,kernel,shape", [("fp32", "ffma", dict(E=80, n=3, A=6, D=20, C=240)),
+                                               ("bf16", "ffma", dict(E=500, n=5, A=11, D=16, C=1000)),
+                                               ("bf16", "pipelined", dict(E=64, n=4, A=8, D=24, C=128))])
+def test_lagged_steps_match_the_oracle(prec, kernel, shape):
+    """Environments that answer after the action (Algorithm 1): every environment runs on its own clock, a call lists
+    those with a new observation and brings the outcome of their previous action."""
+    cfg = workloads.small_config(H=64, L=4, T=26, precision=prec, env=dict(done_thresh24=1 << 22), **shape)
+    E, n, A, T = cfg["E"], cfg["n"], cfg["A"], cfg["T"]
+    w = workloads.make_weights(cfg)
+    obs, avail, rew, done = _env_block(cfg, T)            # [k][e]: the k-th exchange of environment e
+    dev = "cuda:0"
+    actor = binding.Actor(cfg, device=dev, kernel=kernel)
+    actor.set_weights(w)
+    g_acts, g_q = actor.set_trace(T, want_q=True)
+    sess = oracle.Session(cfg, w, np.arange(E))
+    rng = np.random.default_rng(11)
+    k_of = np.zeros(E, np.int64)                          # exchanges each environment has had
+    eps, rtol = 0.1, RTOL[prec]
+    near = greedy = 0
+    for t in range(T):
+        M = E if t == 0 else int(rng.integers(1, E + 1))
+        ids = rng.permutation(E)[:M].astype(np.int32)
+        k = k_of[ids]
+        first = k == 0
+        p_rew = np.where(first, np.float32(7.0), rew[np.maximum(k - 1, 0), ids]).astype(np.float32)
+        p_done = np.where(first, 1, done[np.maximum(k - 1, 0), ids]).astype(np.uint8)   # ignored on a first call
+        o, av = obs[k, ids], avail[k, ids]
+        act = actor.step_lagged(ids, *(torch.as_tensor(x, device=dev) for x in (o, av, p_rew, p_done)), eps).cpu().numpy()
+        tid = torch.as_tensor(ids, device=dev, dtype=torch.long)
+        q_rows = g_q[t].index_select(0, tid).cpu().numpy()
+        _, tr = sess.step_lagged(ids, o, av, p_rew, p_done, eps, adopt=act, trace=("q", "action_free", "explore"))
+        N = M * n
+        re_act, re_ex = oracle.select_batch(q_rows.reshape(N, A), av.reshape(N, A), np.float32(eps), cfg["seed"],
+                                            np.uint32(t), np.repeat(ids.astype(np.uint32), n),
+                                            np.tile(np.arange(n, dtype=np.uint32), M))
+        assert np.array_equal(re_act, act.reshape(N)), f"call {t}"
+        assert np.array_equal(re_ex, tr["explore"].reshape(N))
+        assert row_rel_err(q_rows, tr["q"]).max() <= rtol, f"call {t}"
+        diff = np.argwhere(tr["action_free"] != act)
+        for (x, i) in diff:
+            gap = abs(float(tr["q"][x, i, tr["action_free"][x, i]]) - float(tr["q"][x, i, act[x, i]]))
+            assert gap <= 1e-4 + 2 * rtol * max(float(np.abs(tr["q"][x, i]).max()), 1e-3)
+        near += len(diff)
+        greedy += int((tr["explore"] == 0).sum())
+        k_of[ids] += 1
+    assert near <= max(1, NEAR_TIE_BUDGET[prec] * greedy * 4)
+    torch.cuda.synchronize()
+    st = actor.get_state()
+    for key in ("last_action", "slot", "pos", "ep_count"):
+        assert np.array_equal(st[key].cpu().numpy(), getattr(sess, key)), key
+    assert row_rel_err(st["h"].cpu().numpy(), sess.h).max() <= rtol
+    rv = actor.ring_view()
+    for key in ("slot_epid", "slot_len", "slot_complete"):
+        assert np.array_equal(rv[key].cpu().numpy(), sess.ring[key]), key
+    written = np.arange(cfg["L"])[None, :] < sess.ring["slot_len"][:, None]
+    for key in ("obs", "avail", "action", "reward", "done"):
+        assert np.array_equal(rv[key].cpu().numpy()[written], sess.ring[key][written]), key
+    assert row_rel_err(rv["q"].cpu().numpy()[written], sess.ring["q"][written]).max() <= rtol
+    status, counters = actor.status()
+    oc = sess.counters
+    assert status == 0 and counters["agent_steps"] == oc[oracle.CNT_STEPS]
+    assert counters["episodes"] == oc[oracle.CNT_EPISODES] > 0 and counters["truncated"] == oc[oracle.CNT_TRUNCATED] > 0
+    actor.destroy()

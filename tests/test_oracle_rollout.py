@@ -230,3 +230,63 @@ def test_subset_steps_touch_only_the_listed_environments_and_compose_to_a_full_s
     for k in full.ring:
         assert np.array_equal(full.ring[k], part.ring[k]), k
     assert np.array_equal(full.counters, part.counters)
+
+
+def test_lagged_step_equals_the_synchronous_step_with_outcomes_one_call_late():
+    """Algorithm 1: the reward and the end of the game are known after the action, so they reach the worker with the
+    next observation.  Feeding each outcome one call late gives the same decisions, and every closed episode is
+    recorded exactly as by the synchronous step (same records, same lengths, truncation at the slot length too)."""
+    cfg = workloads.small_config(E=5, C=60, L=4, T=17, env=dict(done_thresh24=1 << 22))
+    E, T = cfg["E"], cfg["T"]
+    sync, _ = _session(cfg)
+    lag, _ = _session(cfg)
+    tr = _roll(sync, cfg)
+    ids = np.arange(E)
+    zr, zd = np.zeros(E, np.float32), np.zeros(E, np.uint8)
+    for t in range(T):
+        eps = oracle.eps_at(cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"], t)
+        acts, ltr = lag.step_lagged(ids, tr["obs"][t], tr["avail"][t], tr["reward"][t - 1] if t else zr,
+                                    tr["done"][t - 1] if t else zd, eps, trace=("q",))
+        assert np.array_equal(acts, tr["action"][t]), t
+        assert np.array_equal(ltr["q"], tr["q"][t]), t
+    closed = lag.ring["slot_complete"] == 1
+    assert closed.sum() >= 8 and (tr["done"].sum() > 0) and sync.counters[oracle.CNT_TRUNCATED] > 0
+    for k in ("obs", "avail", "action", "q", "reward", "done", "slot_epid", "slot_len"):
+        assert np.array_equal(lag.ring[k][closed], sync.ring[k][closed]), k
+    # the synchronous session has also closed the episodes that end with the last step; the lagged one will on its
+    # next call: until then the last outcome is missing and the cursor stands one past the record
+    last_closes = (tr["done"][T - 1] != 0) | (tr["pos"][T - 1] + 1 == cfg["L"])
+    assert np.array_equal(lag.ep_count + last_closes, sync.ep_count)
+    assert np.array_equal(lag.pos[~last_closes], sync.pos[~last_closes])
+
+
+def test_lagged_step_by_hand():
+    """One environment, slot length 3: first call has nothing to commit; a 'done' closes the episode before the
+    decision, which then starts from a zero hidden state and no last action in the next slot."""
+    cfg = workloads.small_config(E=1, C=2, L=3, T=1)
+    sess, w = _session(cfg)
+    n, D, A, H = cfg["n"], cfg["D"], cfg["A"], cfg["H"]
+    rng = np.random.default_rng(5)
+    obs = rng.uniform(-1, 1, size=(5, 1, n, D)).astype(np.float32)
+    avail = np.ones((1, n, A), np.uint8)
+    one = lambda v, dt: np.array([v], dt)
+    sess.step_lagged([0], obs[0], avail, one(9.0, np.float32), one(1, np.uint8), 0.0)       # outcome ignored
+    assert sess.pos[0] == 1 and sess.ep_count[0] == 0 and sess.ring["slot_len"][0] == 1
+    sess.step_lagged([0], obs[1], avail, one(0.5, np.float32), one(0, np.uint8), 0.0)
+    assert sess.pos[0] == 2 and sess.ring["reward"][0, 0] == 0.5 and sess.ring["done"][0, 0] == 0
+    _, tr = sess.step_lagged([0], obs[2], avail, one(-2.0, np.float32), one(1, np.uint8), 0.0, trace=("q",))
+    assert sess.slot[0] == 1 and sess.pos[0] == 1 and sess.ep_count[0] == 1
+    assert list(sess.ring["reward"][0]) == [0.5, -2.0, 0.0] and list(sess.ring["done"][0]) == [0, 1, 0]
+    assert sess.ring["slot_len"][0] == 2 and sess.ring["slot_complete"][0] == 1 and sess.ring["slot_complete"][1] == 0
+    assert sess.ring["slot_epid"][1] == 1 and sess.counters[oracle.CNT_EPISODES] == 1
+    for i in range(n):
+        q0, _ = oracle.agent_forward(cfg, w, obs[2, 0, i], i, -1, np.zeros(H, np.float32))
+        assert np.array_equal(tr["q"][0, i], q0)
+    # two more records fill the slot (length 3); the next call truncates it
+    sess.step_lagged([0], obs[3], avail, one(1.0, np.float32), one(0, np.uint8), 0.0)
+    sess.step_lagged([0], obs[4], avail, one(2.0, np.float32), one(0, np.uint8), 0.0)
+    assert sess.pos[0] == 3 and sess.ring["slot_len"][1] == 3 and sess.ring["slot_complete"][1] == 0
+    sess.step_lagged([0], obs[0], avail, one(3.0, np.float32), one(0, np.uint8), 0.0)
+    assert sess.slot[0] == 0 and sess.pos[0] == 1 and sess.ep_count[0] == 2
+    assert list(sess.ring["reward"][1]) == [1.0, 2.0, 3.0] and sess.ring["slot_complete"][1] == 1
+    assert sess.counters[oracle.CNT_TRUNCATED] == 1 and sess.ring["slot_epid"][0] == 2
