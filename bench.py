@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--subset", type=float, default=0.0, metavar="FRACTION",
                     help="time marl_actor_step_subset instead: every call steps a seeded list of FRACTION * E "
                          "environments (a multiple of four), T calls per step")
+    ap.add_argument("--lagged", action="store_true",
+                    help="with --subset: marl_actor_step_lagged (reward/done are the outcome of the previous action)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sampler", type=int, default=0, metavar="B",
@@ -305,9 +307,11 @@ def run_subset(args, cfg, dev):
     acts = torch.empty((M, n), dtype=torch.int32, device=dev)
     del staged
 
+    step = actor.step_lagged if args.lagged else actor.step_subset
+
     def one_step():
         for k in range(T):
-            actor.step_subset(lists[k % 4], *inputs[k % 4], cfg["eps_start"], acts)
+            step(lists[k % 4], *inputs[k % 4], cfg["eps_start"], acts)
 
     for _ in range(args.warmup):
         one_step()
@@ -332,7 +336,7 @@ def run_subset(args, cfg, dev):
                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
                       "higher_is_better": True, "dtype": cfg["precision"], "data": "synthetic",
                       "config": {"workload": cfg["name"], "E": E, "M": M, "n": n, "T": T, "kernel": actor.kernel_name,
-                                 "step": f"T={T} marl_actor_step_subset calls over lists of M={M} of E={E} environments",
+                                 "step": f"T={T} {'marl_actor_step_lagged' if args.lagged else 'marl_actor_step_subset'} calls over lists of M={M} of E={E} environments",
                                  "l2": f"each call reads {in_bytes / 1e6:.0f} MB of inputs and {M * n * cfg['H'] * 4 / 1e6:.0f} MB of "
                                        "hidden state (four lists in turn)"},
                       "gpu_launches": int(launches),

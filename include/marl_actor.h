@@ -224,7 +224,7 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
  * the slot is full, the episode is closed (header, counters, next slot, zero hidden state, no last action); then
  * the decision on this observation is recorded with reward 0 and done 0 for now.  An environment's first call has
  * nothing waiting: its prev_reward / prev_done are ignored.  Do not mix with the synchronous stepping calls on one
- * actor (they close an episode in the step that ends it).  Runs on the CUDA-core kernel. */
+ * actor (they close an episode in the step that ends it).  Kernel choice as for marl_actor_step_subset. */
 int marl_actor_step_lagged(marl_actor_t* a, const int32_t* env_ids, int32_t M, const float* obs,
                            const uint8_t* avail, const float* prev_reward, const uint8_t* prev_done, float eps,
                            int32_t* actions_out);

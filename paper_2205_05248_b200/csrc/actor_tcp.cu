@@ -199,11 +199,14 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
 }
 
 // PLAIN: the word-by-word path of shapes whose per-environment blocks are not 16-byte multiples.
-// LIST: the call's rows are the environments of p.env_ids (a partial step); inputs, the last step's actions and the
-// tiling follow the row, state, ring cursors, the draw's key and the trace follow the environment.
-template <int NQ, bool PLAIN, bool LIST>
+// MODE 1, 2 (LIST): the call's rows are the environments of p.env_ids (a partial step); inputs, the last step's
+// actions and the tiling follow the row, state, ring cursors, the draw's key and the trace follow the environment.
+// MODE 2 (LAG, one step per launch): reward/done are the outcome of each environment's previous action: they complete
+// the record at pos - 1 and may close the episode BEFORE this step's decision; nothing closes after it.
+template <int NQ, bool PLAIN, int MODE>
 __global__ void __launch_bounds__(TP_THREADS, 1)
     actor_tcp_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TpLayout L) {
+  constexpr bool LIST = MODE >= 1, LAG = MODE == 2;
   extern __shared__ __align__(1024) uint8_t smem[];
   using namespace tc;
   TpBars* B = reinterpret_cast<TpBars*>(smem + L.off_bar);
@@ -384,15 +387,20 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           slot = p.slot[e];
           pos = p.pos[e];
           epc = p.ep_count[e];
-          ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
+          ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L + (LAG ? 1 : 0)) ? 1 : 0;
           done_next = p.done[x];
+          if (LAG && ok && pos > 0 && (done_next || pos == p.L)) {  // the late outcome closes the episode first
+            epc += 1;
+            slot = e * p.S + (int)(epc % p.S);
+            pos = 0;
+          }
         }
         for (int s = 0; s < T; ++s, ++kstep) {
           unsigned long long rec = 0;
           int closes = 0;
           if (mine && ok) {
             rec = reinterpret_cast<unsigned long long>(p.ring + (size_t)slot * p.slot_stride + (size_t)pos * rec_bytes);
-            if (done_next || pos + 1 == p.L) {  // the cursor after this step
+            if (!LAG && (done_next || pos + 1 == p.L)) {  // the cursor after this step
               closes = 1;
               epc += 1;
               slot = e * p.S + (int)(epc % p.S);
@@ -447,10 +455,28 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           slot = p.slot[e];
           pos = p.pos[e];
           epc = p.ep_count[e];
-          ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L) ? 1 : 0;
+          ok = (slot >= 0 && slot < p.E * p.S && pos >= 0 && pos < p.L + (LAG ? 1 : 0)) ? 1 : 0;
           if (!ok) st_bits |= MARL_STATUS_BAD_INDEX;
           reward_next = p.reward[x];
           done_next = p.done[x];
+          if (LAG) {
+            if (ok && pos > 0) {  // the outcome of the previous action completes its record and may close the episode
+              uint8_t* prev = p.ring + (size_t)slot * p.slot_stride + (size_t)(pos - 1) * rec_bytes;
+              *reinterpret_cast<float*>(prev + p.rl.off_reward) = reward_next;
+              prev[p.rl.off_done] = done_next ? 1 : 0;
+              if (done_next || pos == p.L) {
+                p.slot_len[slot] = pos;
+                p.slot_complete[slot] = 1;
+                c_episodes += 1;
+                if (!done_next) c_trunc += 1;
+                epc += 1;
+                slot = e * p.S + (int)(epc % p.S);
+                pos = 0;
+              }
+            }
+            reward_next = 0.f;  // this step's own outcome is not known yet
+            done_next = 0;
+          }
         }
         // Copies the tails of one step (buffer bb, record addresses in tdst_s) to the ring: 16 bytes per lane, the
         // pieces of all environments in one flat loop.
@@ -469,7 +495,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const uint32_t b = it & 1;
           const float reward = reward_next;
           const int done = done_next ? 1 : 0;
-          const int close = (ok && (done || pos + 1 == p.L)) ? 1 : 0;
+          const int close = (!LAG && ok && (done || pos + 1 == p.L)) ? 1 : 0;
           uint8_t* tl = tails + b * tail_set + (uint32_t)lane * L.tail_bytes;
           unsigned long long dst = 0;
           close_s[b * 32 + lane] = close;
@@ -708,10 +734,15 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 
       // ---- tile prologue: hidden state and last actions from global memory ----
       {
+        bool carry = live;  // the row continues an episode
+        if (LAG && live) {  // ... unless the late outcome has just ended it
+          const int ps = p.pos[e];
+          if (ps > 0 && (p.done[e0 + el] || ps == p.L)) carry = false;
+        }
         const float4* src = reinterpret_cast<const float4*>(p.h + grow * TC_H + cb);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          const float4 v = live ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 v = carry ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
           h[4 * q] = v.x; h[4 * q + 1] = v.y; h[4 * q + 2] = v.z; h[4 * q + 3] = v.w;
         }
 #pragma unroll
@@ -721,7 +752,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
         }
         if (half == 0) {
-          la = live ? p.last_action[grow] : -1;
+          la = carry ? p.last_action[grow] : -1;
           if (la >= A) la = -1;
           la_s[row] = la;
         }
@@ -943,15 +974,17 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
   if (L.plain && p.M % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
-  const bool list = p.env_ids != nullptr;
+  const int mode = p.env_ids == nullptr ? 0 : (p.lagged ? 2 : 1);
+  if (p.lagged && (mode != 2 || p.T != 1)) return 0;  // late outcomes: one step per launch over a list
   auto pick = [&](auto nq) {
     constexpr int Q = decltype(nq)::value;
-    return list ? (L.plain ? actor_tcp_kernel<Q, true, true> : actor_tcp_kernel<Q, false, true>)
-                : (L.plain ? actor_tcp_kernel<Q, true, false> : actor_tcp_kernel<Q, false, false>);
+    return mode == 2 ? (L.plain ? actor_tcp_kernel<Q, true, 2> : actor_tcp_kernel<Q, false, 2>)
+         : mode == 1 ? (L.plain ? actor_tcp_kernel<Q, true, 1> : actor_tcp_kernel<Q, false, 1>)
+                     : (L.plain ? actor_tcp_kernel<Q, true, 0> : actor_tcp_kernel<Q, false, 0>);
   };
   auto kernel = L.NQ == 16 ? pick(std::integral_constant<int, 16>()) : pick(std::integral_constant<int, 32>());
-  static uint32_t configured[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + (list ? 4 : 0)];
+  static uint32_t configured[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + 4 * mode];
   if (L.total > conf) {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return -(int)e;

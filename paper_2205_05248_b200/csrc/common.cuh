@@ -67,7 +67,7 @@ struct ActorParams {
   // partial step (FFMA kernel only): the call's rows are the M listed environments; null: all E in order
   const int32_t* env_ids;
   int32_t M;
-  // FFMA kernel, T == 1: reward/done are the outcome of each environment's PREVIOUS action (committed at pos - 1)
+  // T == 1 over a list: reward/done are the outcome of each environment's PREVIOUS action (committed at pos - 1)
   int32_t lagged;
 };
 

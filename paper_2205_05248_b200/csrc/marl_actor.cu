@@ -612,7 +612,7 @@ static int step_list(marl_actor* a, const int32_t* env_ids, int32_t M, const flo
   p.M = M;
   p.lagged = lagged ? 1 : 0;
   int rc = 0;
-  if (a->use_tcp && !lagged) {  // 0: these pointers or this list length cannot be bulk-copied
+  if (a->use_tcp) {  // 0: these pointers or this list length cannot be bulk-copied
     tc_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
     rc = launch_actor_tcp(p, a->sms, a->stream);
   }

@@ -129,7 +129,9 @@ def test_subset_list_is_validated_on_the_host():
 
 @pytest.mark.parametrize("prec,kernel,shape", [("fp32", "ffma", dict(E=80, n=3, A=6, D=20, C=240)),
                                                ("bf16", "ffma", dict(E=500, n=5, A=11, D=16, C=1000)),
-                                               ("bf16", "pipelined", dict(E=64, n=4, A=8, D=24, C=128))])
+                                               ("bf16", "pipelined", dict(E=64, n=4, A=8, D=24, C=128)),
+                                               ("bf16", "pipelined", dict(E=700, n=8, A=14, D=80, C=1400)),
+                                               ("bf16", "pipelined", dict(E=300, n=5, A=12, D=55, C=600))])
 def test_lagged_steps_match_the_oracle(prec, kernel, shape):
     """Environments that answer after the action (Algorithm 1): every environment runs on its own clock, a call lists
     those with a new observation and brings the outcome of their previous action."""
