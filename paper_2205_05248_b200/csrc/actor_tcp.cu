@@ -203,10 +203,14 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
 // actions and the tiling follow the row, state, ring cursors, the draw's key and the trace follow the environment.
 // MODE 2 (LAG, one step per launch): reward/done are the outcome of each environment's previous action: they complete
 // the record at pos - 1 and may close the episode BEFORE this step's decision; nothing closes after it.
+// MODE 3: MODE 0 for launches of a few steps, where the tile-to-tile transition is a large part of the time: the
+// hidden-state rows then move coalesced through a scratch and the next tile's rows are prefetched into L2 (modes 1
+// and 2 do the same).  Launches of many steps keep the shorter transition code: its footprint in the step loop's
+// instruction stream and registers costs them more (1.2 %) than the transition saves.
 template <int NQ, bool PLAIN, int MODE>
 __global__ void __launch_bounds__(TP_THREADS, 1)
     actor_tcp_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TpLayout L) {
-  constexpr bool LIST = MODE >= 1, LAG = MODE == 2;
+  constexpr bool LIST = MODE == 1 || MODE == 2, LAG = MODE == 2, FASTX = MODE != 0;
   extern __shared__ __align__(1024) uint8_t smem[];
   using namespace tc;
   TpBars* B = reinterpret_cast<TpBars*>(smem + L.off_bar);
@@ -721,6 +725,13 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
     unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0;
     uint32_t st_bits = 0, it = 0;
     float h[32];
+    // this thread's half (32 floats) of tile row r's hidden state in global memory
+    auto h_row = [&](int e0, int r) -> float* {
+      if (!LIST) return p.h + ((size_t)e0 * n + (size_t)r) * TC_H + cb;  // a tile's rows are contiguous
+      const int rel = rowenv_s[r];  // r / n
+      const int env = __ldg(p.env_ids + e0 + rel);
+      return p.h + ((size_t)env * n + (size_t)(r - rel * n)) * TC_H + cb;
+    };
 
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int e0 = tile * L.ept;
@@ -734,16 +745,59 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 
       // ---- tile prologue: hidden state and last actions from global memory ----
       {
+        TP_STAMP(tid == 0, it, 22);
         bool carry = live;  // the row continues an episode
         if (LAG && live) {  // ... unless the late outcome has just ended it
           const int ps = p.pos[e];
           if (ps > 0 && (p.done[e0 + el] || ps == p.L)) carry = false;
         }
-        const float4* src = reinterpret_cast<const float4*>(p.h + grow * TC_H + cb);
+        const int la_mem = (carry && half == 0) ? p.last_action[grow] : -1;  // in flight beside the rows below
+        // A thread owns 128 bytes of its row, so a warp reading "its own" pieces would touch 32 lines per
+        // instruction.  The rows go through a warp-private 2 KB scratch instead (the y operand buffer, idle
+        // between tiles): eight lanes fetch one row's 128 bytes, the scratch's piece index is xor-ed with the row so
+        // that neither side has bank conflicts, and each thread then takes its row, 16 rows per pass.
+        if constexpr (FASTX) {
+          uint4* sw = reinterpret_cast<uint4*>(yb) + warp * 128;  // this warp's scratch
+          const int wrow0 = (warp & 3) * 32;                      // first tile row of this warp
+          uint4 f[2][4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const float4 v = carry ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
-          h[4 * q] = v.x; h[4 * q + 1] = v.y; h[4 * q + 2] = v.z; h[4 * q + 3] = v.w;
+          for (int ps = 0; ps < 2; ++ps)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int r = wrow0 + ps * 16 + 4 * j + (lane >> 3);
+              f[ps][j] = make_uint4(0u, 0u, 0u, 0u);
+              if (r < R) f[ps][j] = __ldg(reinterpret_cast<const uint4*>(h_row(e0, r)) + (lane & 7));
+            }
+#pragma unroll
+          for (int ps = 0; ps < 2; ++ps) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int rl = 4 * j + (lane >> 3);
+              sw[rl * 8 + ((lane & 7) ^ (rl & 7))] = f[ps][j];
+            }
+            __syncwarp();
+            if ((lane >> 4) == ps) {
+              const int rl = lane & 15;
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const uint4 v = sw[rl * 8 + (q ^ (rl & 7))];
+                h[4 * q] = __uint_as_float(v.x); h[4 * q + 1] = __uint_as_float(v.y);
+                h[4 * q + 2] = __uint_as_float(v.z); h[4 * q + 3] = __uint_as_float(v.w);
+              }
+            }
+            __syncwarp();
+          }
+          if (!carry) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) h[q] = 0.f;
+          }
+        } else {
+          const float4* src = reinterpret_cast<const float4*>(p.h + grow * TC_H + cb);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 v = carry ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+            h[4 * q] = v.x; h[4 * q + 1] = v.y; h[4 * q + 2] = v.z; h[4 * q + 3] = v.w;
+          }
         }
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
@@ -751,15 +805,29 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
                                      pack_bf16x2(h[8 * cc + 4], h[8 * cc + 5]), pack_bf16x2(h[8 * cc + 6], h[8 * cc + 7]));
           *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
         }
+        TP_STAMP(tid == 0, it, 23);
         if (half == 0) {
-          la = carry ? p.last_action[grow] : -1;
+          la = la_mem;
           if (la >= A) la = -1;
           la_s[row] = la;
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
+        TP_STAMP(tid == 0, it, 24);
         asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s is read by both threads of a row
+        TP_STAMP(tid == 0, it, 25);
         warp_arrive(&B->tiled, lane);
+        // The next tile's hidden state is a first touch of its lines (and often of its page): ask for it now, one
+        // line per thread, so that the next prologue finds it in L2.
+        const int tile_n = tile + (int)gridDim.x;
+        if (FASTX && tile_n < p.num_tiles) {
+          const int e0n = tile_n * L.ept;
+          if (row < min(L.ept, p.M - e0n) * n) {
+            const float* nx = h_row(e0n, row);
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(nx));
+            if (half == 0 && ai == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.last_action + (nx - cb - p.h) / TC_H));
+          }
+        }
       }
 
       for (int s = 0; s < T; ++s) {
@@ -941,12 +1009,33 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
       }
 
       // ---- tile epilogue: state back to global memory ----
-      if (live) {
+      if (is_row) p.last_action[grow] = la;
+      if constexpr (FASTX) {
+        uint4* sw = reinterpret_cast<uint4*>(yb) + warp * 128;
+        const int wrow0 = (warp & 3) * 32;
+#pragma unroll
+      for (int ps = 0; ps < 2; ++ps) {  // the rows leave through the same scratch, coalesced
+        if ((lane >> 4) == ps) {
+          const int rl = lane & 15;
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            sw[rl * 8 + (q ^ (rl & 7))] = make_uint4(__float_as_uint(h[4 * q]), __float_as_uint(h[4 * q + 1]),
+                                                     __float_as_uint(h[4 * q + 2]), __float_as_uint(h[4 * q + 3]));
+        }
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int rl = 4 * j + (lane >> 3), r = wrow0 + ps * 16 + rl;
+          if (r < R) reinterpret_cast<uint4*>(h_row(e0, r))[lane & 7] = sw[rl * 8 + ((lane & 7) ^ (rl & 7))];
+        }
+        __syncwarp();
+      }
+      } else if (live) {
         float4* dsth = reinterpret_cast<float4*>(p.h + grow * TC_H + cb);
 #pragma unroll
         for (int q = 0; q < 8; ++q) dsth[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
       }
-      if (is_row) p.last_action[grow] = la;
+      TP_STAMP(tid == 0, it, 26);
       asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s is rewritten by the next tile's prologue
     }
     if (c_steps) atomicAdd(p.counters + CNT_AGENT_STEPS, c_steps);
@@ -974,16 +1063,17 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
   if (L.plain && p.M % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
-  const int mode = p.env_ids == nullptr ? 0 : (p.lagged ? 2 : 1);
+  const int mode = p.env_ids == nullptr ? (p.T < 8 ? 3 : 0) : (p.lagged ? 2 : 1);
   if (p.lagged && (mode != 2 || p.T != 1)) return 0;  // late outcomes: one step per launch over a list
   auto pick = [&](auto nq) {
     constexpr int Q = decltype(nq)::value;
-    return mode == 2 ? (L.plain ? actor_tcp_kernel<Q, true, 2> : actor_tcp_kernel<Q, false, 2>)
+    return mode == 3 ? (L.plain ? actor_tcp_kernel<Q, true, 3> : actor_tcp_kernel<Q, false, 3>)
+         : mode == 2 ? (L.plain ? actor_tcp_kernel<Q, true, 2> : actor_tcp_kernel<Q, false, 2>)
          : mode == 1 ? (L.plain ? actor_tcp_kernel<Q, true, 1> : actor_tcp_kernel<Q, false, 1>)
                      : (L.plain ? actor_tcp_kernel<Q, true, 0> : actor_tcp_kernel<Q, false, 0>);
   };
   auto kernel = L.NQ == 16 ? pick(std::integral_constant<int, 16>()) : pick(std::integral_constant<int, 32>());
-  static uint32_t configured[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  static uint32_t configured[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + 4 * mode];
   if (L.total > conf) {
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
