@@ -843,11 +843,14 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           // an episode that just ended has no last action
           int last = (s > 0 && close_s[(b ^ 1u) * 32 + el]) ? -1 : la_s[row];
           const float* tlr = tab_la + (last >= 0 ? last : 0) * TC_TAB + cb;
+          // both halves of the thread's 32 columns are requested before the one wait
+          uint32_t v2[2][16];
+          tmem_ld16(tmem + lane_addr + TM_FC1 + cb, v2[0]);
+          tmem_ld16(tmem + lane_addr + TM_FC1 + cb + 16, v2[1]);
+          tmem_ld_wait();
 #pragma unroll
           for (int c16 = 0; c16 < 2; ++c16) {
-            uint32_t v[16];
-            tmem_ld16(tmem + lane_addr + TM_FC1 + cb + c16 * 16, v);
-            tmem_ld_wait();
+            uint32_t(&v)[16] = v2[c16];
             float y[16];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
