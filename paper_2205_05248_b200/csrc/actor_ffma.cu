@@ -15,6 +15,7 @@
 // Weights are read through the read-only path from k-major copies, so a warp's load of four output
 // columns for one k is one contiguous 256-byte segment.
 #include "common.cuh"
+#include "launch_util.cuh"
 
 namespace marl {
 
@@ -518,12 +519,10 @@ size_t ffma_smem_bytes(int n, int D, int A, int H) { return ffma_smem_layout(n, 
 int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream) {
   const FfmaSmem sl = ffma_smem_layout(p.n, p.D, p.A, p.H);
   auto kernel = sl.wsmem ? actor_ffma_kernel<true> : actor_ffma_kernel<false>;
-  static size_t configured[2] = {0, 0};
-  size_t& conf = configured[sl.wsmem];
-  if (sl.total > conf) {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.total);
+  static uint32_t configured[2][SMEM_OPTIN_DEVICES];
+  {
+    const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (uint32_t)sl.total, configured[sl.wsmem ? 1 : 0]);
     if (e != cudaSuccess) return -(int)e;
-    conf = sl.total;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;

@@ -29,6 +29,7 @@
 
 #include "actor_tc_layout.cuh"
 #include "common.cuh"
+#include "launch_util.cuh"
 #include "tcgen05.cuh"
 
 namespace marl {
@@ -706,12 +707,10 @@ int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream) {
   // aligned; otherwise the row threads fetch them one step ahead
   L.avail_bulk = ((p.n * p.A) % 16 == 0 && reinterpret_cast<uintptr_t>(p.avail) % 16 == 0) ? 1 : 0;
   auto kernel = L.NQ == 16 ? actor_tc_kernel<16> : actor_tc_kernel<32>;
-  static uint32_t configured[2] = {0, 0};
-  uint32_t& conf = configured[L.NQ == 16 ? 0 : 1];
-  if (L.total > conf) {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+  static uint32_t configured[2][SMEM_OPTIN_DEVICES];
+  {
+    const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L.total, configured[L.NQ == 16 ? 0 : 1]);
     if (e != cudaSuccess) return -(int)e;
-    conf = L.total;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;

@@ -34,6 +34,7 @@
 
 #include "actor_tc_layout.cuh"
 #include "common.cuh"
+#include "launch_util.cuh"
 #include "tcgen05.cuh"
 
 namespace marl {
@@ -1076,12 +1077,11 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
                      : (L.plain ? actor_tcp_kernel<Q, true, 0> : actor_tcp_kernel<Q, false, 0>);
   };
   auto kernel = L.NQ == 16 ? pick(std::integral_constant<int, 16>()) : pick(std::integral_constant<int, 32>());
-  static uint32_t configured[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  uint32_t& conf = configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + 4 * mode];
-  if (L.total > conf) {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+  static uint32_t configured[16][SMEM_OPTIN_DEVICES];
+  {
+    const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L.total,
+                                              configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + 4 * mode]);
     if (e != cudaSuccess) return -(int)e;
-    conf = L.total;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;
