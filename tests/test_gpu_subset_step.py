@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2205_05248_b200 import binding, workloads
-from referee import NEAR_TIE_BUDGET, RTOL, row_rel_err
+from referee import NEAR_TIE_BUDGET, RTOL, row_rel_err, sample_envs
 
 pytestmark = pytest.mark.gpu
 
@@ -191,4 +191,96 @@ def test_lagged_steps_match_the_oracle(prec, kernel, shape):
     oc = sess.counters
     assert status == 0 and counters["agent_steps"] == oc[oracle.CNT_STEPS]
     assert counters["episodes"] == oc[oracle.CNT_EPISODES] > 0 and counters["truncated"] == oc[oracle.CNT_TRUNCATED] > 0
+    actor.destroy()
+
+
+@pytest.mark.parametrize("lagged", [False, True])
+def test_list_steps_full_size_bench_configuration(lagged):
+    """The workload and launch configuration that `bench.py --subset 0.5 [--lagged]` times (E=65536, lists of 32768
+    environments, 20 GB ring, pipelined tensor-core kernel in list mode): the oracle recomputes a seeded sample of
+    environments, each on its own clock, through every call that lists it."""
+    cfg = workloads.config(5)
+    E, n, A, D = cfg["E"], cfg["n"], cfg["A"], cfg["D"]
+    calls, M, eps = 6, E // 2, 0.05
+    w = workloads.make_weights(cfg)
+    dev = "cuda:0"
+    actor = binding.Actor(cfg, device=dev, kernel="auto", work_steps=1)
+    assert actor.kernel_name == "tcgen05-pipelined"
+    actor.set_weights(w)
+    g_acts, g_q = actor.set_trace(calls, want_q=True)
+    staged = actor.env_generate(cfg["env"], 0, calls)                    # [k][e]: the k-th exchange of environment e
+    sample = sample_envs(E, 24, seed=9)
+    where = {int(e): x for x, e in enumerate(sample)}
+    o_obs, o_avail = np.zeros((calls, len(sample), n, D), np.float32), np.zeros((calls, len(sample), n, A), np.uint8)
+    o_rew, o_done = np.zeros((calls, len(sample)), np.float32), np.zeros((calls, len(sample)), np.uint8)
+    for k in range(calls):
+        for x, e in enumerate(sample):
+            o_obs[k, x], o_avail[k, x], o_rew[k, x], o_done[k, x] = oracle.env_emit(cfg, cfg["env"], k, int(e))
+    sess = oracle.Session(cfg, w, sample)
+    rng = np.random.default_rng(3)
+    k_of = np.zeros(E, np.int64)
+    rtol = RTOL[cfg["precision"]]
+    rows = near = listed = 0
+    for t in range(calls):
+        ids = rng.permutation(E)[:M].astype(np.int32)
+        if t % 2 == 0:                                                    # the sample is listed often
+            ids[: len(sample)] = rng.permutation(sample)
+        ids = np.array(list(dict.fromkeys(ids.tolist())), np.int32)       # no environment twice
+        ids = ids[: len(ids) // 4 * 4]
+        listed += len(ids)
+        tid = torch.as_tensor(ids, device=dev, dtype=torch.long)
+        k = torch.as_tensor(k_of[ids], device=dev)
+        km1 = torch.clamp(k - 1, min=0)
+        if lagged:
+            rew = torch.where(k > 0, staged[2][km1, tid], torch.zeros_like(staged[2][0, tid]))
+            done = torch.where(k > 0, staged[3][km1, tid], torch.zeros_like(staged[3][0, tid]))
+            act = actor.step_lagged(ids, staged[0][k, tid].contiguous(), staged[1][k, tid].contiguous(), rew.contiguous(),
+                                    done.contiguous(), eps)
+        else:
+            act = actor.step_subset(ids, staged[0][k, tid].contiguous(), staged[1][k, tid].contiguous(),
+                                    staged[2][k, tid].contiguous(), staged[3][k, tid].contiguous(), eps)
+        pick = np.nonzero(np.isin(ids, sample))[0]                        # rows of the call that the oracle follows
+        s_ids = ids[pick]
+        sx = np.array([where[int(e)] for e in s_ids])
+        ks = k_of[s_ids]
+        act_s = act[torch.as_tensor(pick, device=dev)].cpu().numpy()
+        q_s = g_q[t].index_select(0, torch.as_tensor(s_ids, device=dev, dtype=torch.long)).cpu().numpy()
+        if lagged:
+            p_r = np.where(ks > 0, o_rew[np.maximum(ks - 1, 0), sx], 0).astype(np.float32)
+            p_d = np.where(ks > 0, o_done[np.maximum(ks - 1, 0), sx], 0).astype(np.uint8)
+            _, tr = sess.step_lagged(s_ids, o_obs[ks, sx], o_avail[ks, sx], p_r, p_d, eps, adopt=act_s,
+                                     trace=("q", "action_free", "explore"))
+        else:
+            _, tr = sess.step_subset(s_ids, o_obs[ks, sx], o_avail[ks, sx], o_rew[ks, sx], o_done[ks, sx], eps, adopt=act_s,
+                                     trace=("q", "action_free", "explore"))
+        N = len(s_ids) * n
+        re_act, _ = oracle.select_batch(q_s.reshape(N, A), o_avail[ks, sx].reshape(N, A), np.float32(eps), cfg["seed"],
+                                        np.uint32(t), np.repeat(s_ids.astype(np.uint32), n),
+                                        np.tile(np.arange(n, dtype=np.uint32), len(s_ids)))
+        assert np.array_equal(re_act, act_s.reshape(N)), f"call {t}"
+        assert row_rel_err(q_s, tr["q"]).max() <= rtol, f"call {t}"
+        near += int((tr["action_free"] != act_s).sum())
+        rows += N
+        # the whole call: every chosen action is available
+        chosen = torch.gather(staged[1][k, tid], 2, act.unsqueeze(-1).long()).squeeze(-1)
+        assert bool((chosen == 1).all())
+        k_of[ids] += 1
+    assert rows >= 24 * n * 3 and near <= 3
+    torch.cuda.synchronize()
+    st = actor.get_state()
+    ts = torch.as_tensor(sample, device=dev, dtype=torch.long)
+    for key in ("last_action", "slot", "pos", "ep_count"):
+        assert np.array_equal(st[key].index_select(0, ts).cpu().numpy(), getattr(sess, key)), key
+    assert row_rel_err(st["h"].index_select(0, ts).cpu().numpy(), sess.h).max() <= rtol
+    rv = actor.ring_view()
+    S = sess.S
+    slots = torch.as_tensor((sample[:, None] * S + np.arange(S)[None, :]).reshape(-1), device=dev, dtype=torch.long)
+    for key in ("slot_epid", "slot_len", "slot_complete"):
+        assert np.array_equal(rv[key].index_select(0, slots).cpu().numpy(), sess.ring[key]), key
+    written = np.arange(cfg["L"])[None, :] < sess.ring["slot_len"][:, None]
+    for key in ("obs", "avail", "action", "reward", "done"):
+        assert np.array_equal(rv[key].index_select(0, slots).cpu().numpy()[written], sess.ring[key][written]), key
+    status, counters = actor.status()
+    assert status == 0 and counters["agent_steps"] == listed * n
+    del staged, g_acts, g_q
     actor.destroy()
