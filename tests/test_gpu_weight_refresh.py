@@ -88,3 +88,29 @@ def test_publication_rules():
     torch.cuda.synchronize()
     assert actor.status()[0] == 0
     actor.destroy()
+
+
+def test_published_weights_full_size_bench_configuration():
+    """The configuration `bench.py --refresh` times: workload 5 at full size, one staged 64-step rollout with a
+    publication that takes effect 32 steps in (two launches of 32 steps); the oracle recomputes sampled environments
+    with the same switch."""
+    cfg = workloads.config(5)
+    T = cfg["T"]
+    w0 = workloads.make_weights(cfg)
+    w1 = workloads.make_weights(cfg, seed=cfg["seed"] + 1)
+    actor = binding.Actor(cfg, kernel="auto", work_steps=1)
+    assert actor.kernel_name == "tcgen05-pipelined"
+    actor.set_weights(w0, version=1)
+    acts, q = actor.set_trace(T, want_q=True)
+    staged = actor.env_generate(cfg["env"], 0, T)
+    launches = actor.launch_count
+    actor.publish_weights(w1, version=2, effective_step=T // 2)
+    actor.rollout_staged(*staged, T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
+    torch.cuda.synchronize()
+    assert actor.launch_count - launches == 2 and actor.weights_version == 2
+    res = referee(cfg, w0, actor, acts, q, env_ids=sample_envs(cfg["E"], 24, seed=6), weight_schedule=[(T // 2, w1)])
+    print(f"cfg5 full size with a publication: {res}")
+    status, counters = actor.status()
+    assert status == 0 and counters["agent_steps"] == cfg["E"] * cfg["n"] * T
+    del staged, acts, q
+    actor.destroy()
