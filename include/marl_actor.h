@@ -217,8 +217,8 @@ int marl_actor_step_subset(marl_actor_t* a, const int32_t* env_ids, int32_t M, c
                            const uint8_t* avail, const float* reward, const uint8_t* done, float eps,
                            int32_t* actions_out);
 
-/* marl_actor_step_subset for environments that answer after the action (Algorithm 1: put o, get a, then
- * "o, r <- Env.step(a)"): prev_reward f32[M] and prev_done u8[M] (device) are the outcome of each listed
+/* marl_actor_step_subset for environments that answer after the action (Algorithm 1: the actor sends its
+ * observation, receives the action and only then steps the environment): prev_reward f32[M] and prev_done u8[M] (device) are the outcome of each listed
  * environment's PREVIOUS action and arrive with this observation.  Per environment, in this order: if a record of
  * the open episode waits for its outcome (cursor > 0), the outcome is written into it and, if the game ended or
  * the slot is full, the episode is closed (header, counters, next slot, zero hidden state, no last action); then
@@ -282,7 +282,7 @@ int marl_actor_set_trace(marl_actor_t* a, int32_t* actions, float* q, int32_t ca
 
 int marl_ring_view(const marl_actor_t* a, marl_ring_view_t* out);
 
-/* The learner's read of the pool (Algorithm 3, "randomly sample B samples from the experience replay pool"; the
+/* The learner's read of the pool (Algorithm 3: the learner draws a batch of B samples at random from the replay pool; the
  * paper fixes neither the unit nor the law of a sample).  A sample is one complete episode, drawn uniformly and
  * with replacement among the slots whose episode is closed: batch element b of draw number draw_index makes up to
  * MARL_SAMPLE_ATTEMPTS attempts; attempt a takes word 0 of the Philox4x32-10 block with counter

@@ -365,8 +365,8 @@ SAMPLE_ATTEMPTS = 16  # draws per batch element before it is reported empty
 
 
 def ring_sample(ring: dict, seed: int, draw_index: int, B: int) -> dict:
-    """The learner's draw of B episodes from the replay pool (Algorithm 3: "randomly sample B samples from the
-    experience replay pool"), written out plainly.
+    """The learner's draw of B episodes from the replay pool (Algorithm 3: the learner draws a batch of B samples at
+    random from the pool), written out plainly.
 
     The paper fixes neither the law nor the unit of a sample; the reading taken here: a sample is one complete
     episode, drawn uniformly and with replacement among the slots whose episode is closed.  Batch element b of

@@ -524,8 +524,8 @@ void oracle_step(const oracle_dims* d, const oracle_weights* w, const int32_t* e
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The same step when the environment answers after the action (Algorithm 1: put o, get a, then
-// "o, r <- Env.step(a)"): the reward and the end-of-game flag of an action reach the worker with the NEXT
+// The same step when the environment answers after the action (Algorithm 1: the actor sends its observation,
+// receives the action and only then steps the environment): the reward and the end-of-game flag of an action reach the worker with the NEXT
 // observation of that environment.  For each listed environment, in this order:
 //   1. if a record of the open episode is still waiting for its outcome (pos > 0): prev_reward / prev_done
 //      are written into that record (pos - 1); if the game ended, or the slot is full (pos == L), the

@@ -2,7 +2,7 @@
 
 * hidden state is private to one (environment, agent) pair (Sec. III-A, Fig. 3);
 * an episode end resets the environment's recurrent state (Algorithm 1: reset at episode start);
-* every step is recorded and whole episodes are handed over (Algorithm 1, last lines of the loop).
+* every step is recorded and whole episodes are handed over (Algorithm 1).
 """
 import numpy as np
 
