@@ -123,6 +123,12 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   int ns = (int)(room / (L.chunk_bytes + L.rs_bytes));
   if (ns > TP_MAX_STAGES) ns = TP_MAX_STAGES;
   if (ns < 0) ns = 0;
+  // A converter warp waits for "the other phase" of a slot's barrier, which reads as complete while the slot's
+  // previous chunk has not even arrived.  That previous chunk must therefore be behind the waiter in program order:
+  // either it belongs to an earlier step (the ring holds a whole tile-step of chunks), or the same warp converts it
+  // (a converter warp takes every fourth chunk, so the ring length is a multiple of four).
+  const int nck_max = (L.ept + TP_G - 1) / TP_G;
+  if (ns < nck_max) ns = ns / (TP_CONV / 32) * (TP_CONV / 32);
   L.NS = ns;
   L.off_rstage = o + (uint32_t)ns * L.chunk_bytes + 32;  // (+32: the mask words read a few bytes past a row)
   L.total = L.off_rstage + (uint32_t)ns * L.rs_bytes;
@@ -136,7 +142,7 @@ bool tcp_supported(int n, int D, int A, int H, int prec) {
   if (D < 1 || D > 256 || n < 4 || n > 32 || A < 1 || A > 32) return false;
   if ((n * A) % 4 != 0) return false;  // a chunk's availability bytes must be a 16-byte multiple
   const TpLayout L = tp_layout(n, D, A, rec_bytes_of(n, D, A));
-  // two tile-steps of chunks in flight at least, so that loads run well ahead of the network
+  // enough staging for loads to run ahead of the network (tp_layout leaves 0 where the ring would be unsafe)
   return L.ept >= TP_G && L.NS >= 3 && L.total <= TC_SMEM_MAX;
 }
 

@@ -409,3 +409,55 @@ def test_pipelined_kernel_falls_back_on_unaligned_inputs():
     assert a2.shape == a1.shape and pipe.status()[0] == 0
     for a in (pipe, tens, ffma):
         a.destroy()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_pipelined_kernel_seeded_shapes(seed):
+    """Seeded shapes inside the pipelined kernel's stated domain (4..32 agents, 1..32 actions with n * A a multiple of
+    four, 1..256 observation features): environment counts that leave ragged tiles and partial chunks, short and
+    long slots, single-step and multi-step launches mixed.  Each is refereed against the oracle on every row."""
+    rng = np.random.default_rng(1000 + seed)
+    done_shapes = 0
+    while done_shapes < 4:
+        n = int(rng.integers(4, 33))
+        A = int(rng.integers(1, 33))
+        if (n * A) % 4:
+            continue
+        D = int(rng.integers(1, 257))
+        tile_envs = max(1, 128 // n)
+        E = int(rng.integers(1, 4 * tile_envs + 3))
+        L = int(rng.integers(2, 9))
+        T = int(rng.integers(6, 15))
+        cfg = workloads.small_config(H=64, precision="bf16", n=n, A=A, D=D, E=E, C=E * int(rng.integers(1, 3)), L=L, T=T,
+                                     seed=workloads.SEED_BASE + 500 + 10 * seed + done_shapes,
+                                     env=dict(done_thresh24=int(rng.integers(0, 1 << 22))))
+        try:
+            actor = binding.Actor(cfg, kernel="pipelined")
+        except binding.MarlError:
+            continue                                  # outside the kernel's shared-memory budget: not its domain
+        actor.destroy()
+        w = workloads.make_weights(cfg)
+        cut = int(rng.integers(1, T))
+        splits = [cut, T - cut] if rng.integers(0, 2) else [1] * 2 + [T - 2]
+        print(f"n={n} A={A} D={D} E={E} C={cfg['C']} L={L} T={T} splits={splits} done_thresh24={cfg['env']['done_thresh24']}", flush=True)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="pipelined", splits=splits)
+        assert actor.kernel_name == "tcgen05-pipelined"
+        res = referee(cfg, w, actor, acts, q, near_tie_budget=4e-3)
+        print(f"   {res}")
+        actor.destroy()
+        done_shapes += 1
+
+
+def test_shape_with_a_short_staging_ring_leaves_the_pipelined_kernel():
+    """n=8, D=81, A=11 leaves room for three staging slots but a tile-step has four chunks: a converter warp would wait
+    on a slot whose previous chunk belongs to another warp of the same step.  The pipelined kernel must not take the
+    shape (it once did, and read stale availability bytes); the other kernels do."""
+    cfg = workloads.small_config(H=64, precision="bf16", n=8, A=11, D=81, E=40, C=80, L=6, T=6,
+                                 env=dict(done_thresh24=2578527))
+    with pytest.raises(binding.MarlError):
+        binding.Actor(cfg, kernel="pipelined")
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w, kernel="auto", splits=[5, 1])
+    assert actor.kernel_name != "tcgen05-pipelined"
+    referee(cfg, w, actor, acts, q, near_tie_budget=4e-3)
+    actor.destroy()
