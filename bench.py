@@ -55,6 +55,9 @@ def parse_args():
                     help="with --subset: marl_actor_step_lagged (reward/done are the outcome of the previous action)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--crossover", action="store_true",
+                    help="time the CUDA-core, one-tile and pipelined kernels on the same bf16 rollouts over a range of "
+                         "batch sizes (E x n rows from 24 to 16384): the evidence behind the automatic kernel choice")
     ap.add_argument("--sampler", type=int, default=0, metavar="B",
                     help="measure the learner-side episode sampler instead: draws of B episodes from a filled ring")
     return ap.parse_args()
@@ -284,6 +287,50 @@ def run_sampler(args, cfg, dev):
     actor.destroy()
 
 
+def run_crossover(args, dev):
+    """--crossover: one rollout of T=32 steps per launch, bf16, on the 3-agent and the 8-agent shapes, for every
+    kernel that takes the shape, over batch sizes from one partial tile to many waves.  Each launch is timed with
+    its own event pair; the median of the repetitions is reported in microseconds per environment step.  (The
+    3-agent, 30-feature shape of the smallest experiment is taken by the CUDA-core kernel only.)"""
+    import torch
+    from paper_2205_05248_b200 import binding, workloads
+    T, reps = 32, max(10, args.steps)
+    rows_list = [24, 48, 96, 192, 384, 768, 1536, 3072, 6144, 16384]
+    table = []
+    for shape in (dict(n=3, D=30, A=9), dict(n=4, D=32, A=8), dict(n=8, D=80, A=14), dict(n=5, D=80, A=11)):
+        for rows in rows_list:
+            E = max(1, rows // shape["n"])
+            cfg = workloads.small_config(H=64, precision="bf16", E=E, C=E, L=64, T=T, **shape)
+            weights = workloads.make_weights(cfg)
+            entry = {"n": shape["n"], "D": shape["D"], "A": shape["A"], "E": E, "rows": E * shape["n"]}
+            for kernel in ("ffma", "tensor", "pipelined"):
+                try:
+                    actor = binding.Actor(cfg, device=str(dev), kernel=kernel, work_steps=1)
+                except binding.MarlError:
+                    entry[kernel] = None          # the kernel does not take this shape
+                    continue
+                actor.set_weights(weights)
+                staged = actor.env_generate(cfg["env"], 0, T)
+                for _ in range(3):
+                    actor.rollout_staged(*staged, T, 0.05)
+                torch.cuda.synchronize()
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+                ev[0].record()
+                for k in range(reps):
+                    actor.rollout_staged(*staged, T, 0.05)
+                    ev[k + 1].record()
+                torch.cuda.synchronize()
+                assert actor.status()[0] == 0
+                per = sorted(ev[k].elapsed_time(ev[k + 1]) for k in range(reps))
+                entry[kernel] = round(1e3 * per[len(per) // 2] / T, 3)
+                actor.destroy()
+                del staged
+            table.append(entry)
+    print(json.dumps({"metric": "microseconds per environment step (median launch of T=32 steps), by kernel and batch",
+                      "unit": "us/step", "higher_is_better": False, "dtype": "bf16", "data": "synthetic", "steps": reps,
+                      "table": table}), flush=True)
+
+
 def run_subset(args, cfg, dev):
     """--subset FRACTION: T calls of marl_actor_step_subset per step, each over one of four seeded lists of
     M = FRACTION * E environments in random order, the dense inputs of each list resident in HBM beforehand.
@@ -366,6 +413,10 @@ def main():
         if rank == 0:
             run_sampler(args, cfg, dev)
         return
+    if args.crossover:
+        if rank == 0:
+            run_crossover(args, dev)
+        return
     if args.subset > 0:
         if rank == 0:
             run_subset(args, cfg, dev)
@@ -399,20 +450,21 @@ def main():
     sampler.start()
     time.sleep(0.25)
     launches0 = actor.launch_count
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]   # one pair per step
     dist_barrier(world)
     torch.cuda.synchronize()
     t_begin = time.perf_counter()
-    ev0.record()
-    for _ in range(args.steps):
+    evs[0].record()
+    for k in range(args.steps):
         one_step()
-    ev1.record()
+        evs[k + 1].record()
     torch.cuda.synchronize()
     t_end = time.perf_counter()
     dist_barrier(world)
     clocks = sampler.stop(t_begin, t_end)
     launches = actor.launch_count - launches0
-    ms_local = ev0.elapsed_time(ev1)
+    ms_local = evs[0].elapsed_time(evs[-1])
+    ms_median = statistics.median(evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps))
     ms_total = dist_max(ms_local, world)
     status, counters = actor.status()
     assert status == 0, f"device status {status}"
@@ -441,8 +493,8 @@ def main():
                     "tflops_effective": flop_rate}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic",
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "ms_per_step_median": ms_median,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic",
             "config": {"workload": cfg["name"], "E": E, "n": n, "D": cfg["D"], "A": cfg["A"], "H": cfg["H"], "T": T,
                        "ring": f"{cfg['C']}x{cfg['L']}", "kernel": actor.kernel_name,
                        "step": f"one marl_rollout_staged call = T={T} environment steps over E={E} environments",

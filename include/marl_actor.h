@@ -4,7 +4,7 @@
  * What the library does.  A "worker" in the actor-worker-learner framework (Sec. III-B, Algorithm 2)
  * repeats: get the observations of all of its environments, decide with the shared policy network, send
  * the actions back.  Each environment step is recorded and whole episodes are handed to the learner's
- * replay pool (Algorithm 1; Algorithm 3, "store it in the experience replay pool").  The hidden state of
+ * replay pool (Algorithm 1 for the hand-over, Algorithm 3 for the learner's side of it).  The hidden state of
  * the recurrent agent is kept per (environment, agent) and never mixed across environments (Sec. III-A,
  * Fig. 3).  This library is that loop for E environments x n agents on the GPU:
  *
@@ -76,7 +76,7 @@ typedef struct {
   int32_t n_agents;      /* n in [1, 32] */
   int32_t obs_dim;       /* D in [1, 512] */
   int32_t n_actions;     /* A in [1, 32] */
-  int32_t hidden;        /* H in {32, 64, 96, 128} */
+  int32_t hidden;        /* H in {64, 128} */
   int32_t ring_episodes; /* C: episode slots of the replay ring, a positive multiple of E */
   int32_t ring_steps;    /* L: steps per slot; an episode reaching L steps is truncated */
   int32_t precision;     /* MARL_PRECISION_* */
@@ -173,7 +173,7 @@ int marl_actor_query_sizes(const marl_actor_config_t* cfg, marl_actor_sizes_t* o
  * Fails with MARL_ECUDA if no CUDA device is usable: there is no CPU path. */
 int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out);
 
-/* Loads the network (Algorithm 2: "get parameters from the shared memory pool").  HOST fp32 arrays in
+/* Loads the network (Algorithm 2: an iteration starts by fetching the current parameters).  HOST fp32 arrays in
  * [out][in] layout, copied and repacked before the call returns to the caller's stream order:
  *   W1 [H][D+n+A], b1 [H], W_ih [3H][H], b_ih [3H], W_hh [3H][H], b_hh [3H] (row blocks r|z|n),
  *   W2 [A][H], b2 [A].  In bf16 precision the four matrices are rounded to bf16 (RNE); biases stay fp32.
@@ -259,16 +259,19 @@ int marl_rollout(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double
  * device memory - programs that gave all of it to their own pool at start-up, or that must avoid cudaMalloc
  * because it synchronises the device and may fail in the middle of a run.  Same arguments and same results as
  * marl_rollout, but the staging window for the generated environment steps is a fixed array of
- * MARL_NOALLOC_SCRATCH_BYTES inside the library image instead of the actor's work buffer; the call performs
- * no cudaMalloc, cudaFree or other allocating call.  (Create the actor on caller-provided ring, state and work
+ * MARL_NOALLOC_SCRATCH_BYTES inside the library image instead of the actor's work buffer; the function calls no
+ * cudaMalloc, cudaFree or other allocating routine.  (Create the actor on caller-provided ring, state and work
  * buffers, otherwise marl_actor_create has already allocated.)
- *   - every GPU that loads the library holds the array until the process exits;
+ *   - SET-UP: CUDA loads a library image piece by piece on first use, so the driver places the array on a GPU -
+ *     taking that much of its memory until the process exits - during the FIRST call of this function with that
+ *     GPU current.  Make that call at start-up, before the remaining device memory goes to your pool and outside
+ *     stream capture (the address look-up synchronises); T = 0 does the set-up alone (a and env may be NULL).
+ *     Later calls on the device leave the amount of free device memory unchanged;
  *   - MARL_ENOMEM if one environment step of staging (E*n*(4D+A) + 5E bytes plus alignment) exceeds the
  *     array; longer rollouts run in several windows;
  *   - the array is shared by all actors and calls on a device and keeps the previous call's bytes; nothing
  *     in it needs clearing, since each window is fully rewritten before it is read, but calls whose GPU work
- *     overlaps race on it - serialise them;
- *   - the first call on a device looks up the array's device address; make that call outside stream capture.
+ *     overlaps race on it - serialise them.
  * The actor's device must be current, as for every other call.  Error text is not set for the size and
  * look-up failures of this function itself; the return code tells them apart. */
 #define MARL_NOALLOC_SCRATCH_BYTES (32u << 20)

@@ -12,7 +12,7 @@
 //   * Hidden state: one vector per (environment, agent), never mixed across environments
 //     (Sec. III-A, Fig. 3).
 //   * Replay pool: every step is recorded and whole episodes become visible to the learner
-//     (Sec. III-B, Algorithm 1 "send the collected whole track", Algorithm 3 "store in the pool").
+//     (Sec. III-B; Algorithm 1 hands the finished track over, Algorithm 3 files it in the pool).
 //   * The paper does not print the agent network (it only says "value-based"/Qmix, Sec. III and
 //     Sec. IV-B).  The network here is the usual recurrent Qmix agent:
 //       x = [obs | one-hot(agent id) | one-hot(last action)]  ->  Linear(H) -> ReLU -> GRUCell(H)

@@ -21,6 +21,12 @@ PRECISION = {"fp32": 0, "bf16": 1}
 KERNEL = {"auto": 0, "ffma": 1, "tensor": 2, "pipelined": 3}
 STATUS_NO_AVAIL, STATUS_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4
 
+# Debug aid: with GUARD_BYTES > 0 (a multiple of 256; the test-suite sets it) every buffer an Actor hands to the
+# library gets that many guard bytes of a fixed pattern in front of it and behind it, and ``Actor.check_guards``
+# (called by ``destroy``) raises if the library has written outside a buffer.
+GUARD_BYTES = 0
+GUARD_PATTERN = 0xA5
+
 EXPORTS = [
     "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_publish_weights",
     "marl_actor_weights_version",
@@ -194,9 +200,22 @@ class Actor:
         steps = max(1, min(steps, (work_budget_bytes - sizes["work_bytes_min"]) // per + 1))
         wbytes = sizes["work_bytes_min"] + (steps - 1) * per
         u8 = dict(dtype=torch.uint8, device=self.device)
-        self.ring_mem = torch.zeros(sizes["ring_bytes"], **u8)   # padding bytes are never written
-        self.state_mem = torch.empty(sizes["state_bytes"], **u8)
-        self.work_mem = torch.empty(wbytes, **u8)
+        self._guards = []
+
+        def alloc(nbytes, zero):
+            g = GUARD_BYTES
+            if g <= 0:
+                return torch.zeros(nbytes, **u8) if zero else torch.empty(nbytes, **u8)
+            assert g % 256 == 0
+            full = torch.zeros(nbytes + 2 * g, **u8) if zero else torch.empty(nbytes + 2 * g, **u8)
+            full[:g] = GUARD_PATTERN
+            full[g + nbytes:] = GUARD_PATTERN
+            self._guards.append((full, g, nbytes))
+            return full[g:g + nbytes]
+
+        self.ring_mem = alloc(sizes["ring_bytes"], True)   # padding bytes are never written
+        self.state_mem = alloc(sizes["state_bytes"], False)
+        self.work_mem = alloc(wbytes, False)
         c = make_config(cfg, kernel)
         self.stream = torch.cuda.current_stream(self.device)
         c.stream = self.stream.cuda_stream
@@ -212,8 +231,17 @@ class Actor:
     # -- lifetime ---------------------------------------------------------------------------------
     def destroy(self):
         if getattr(self, "handle", None):
-            self.lib.marl_actor_destroy(self.handle)
+            self.lib.marl_actor_destroy(self.handle)      # synchronises the stream
             self.handle = None
+            self.check_guards()
+
+    def check_guards(self):
+        """Raises if any guard byte around the ring, state or work buffer has changed (GUARD_BYTES > 0 only)."""
+        for name, (full, g, nbytes) in zip(("ring_mem", "state_mem", "work_mem"), getattr(self, "_guards", [])):
+            front_ok = bool((full[:g] == GUARD_PATTERN).all())
+            back_ok = bool((full[g + nbytes:] == GUARD_PATTERN).all())
+            if not (front_ok and back_ok):
+                raise MarlError(f"the library wrote outside {name} ({'before' if not front_ok else 'behind'} the buffer)")
 
     def __del__(self):
         try:

@@ -191,6 +191,11 @@ struct marl_actor {
   bool image_free_recorded, pending;
   uint64_t pending_version, pending_step;
   std::vector<uint8_t> id_seen;  // scratch of marl_actor_step_subset
+  // pinned staging of the environment list, two buffers in turn, each with the event of its last upload
+  int32_t* ids_host[2];
+  cudaEvent_t ids_copied[2];
+  bool ids_in_flight[2];
+  int ids_next;
   uint8_t* host_pack2;  // pinned, so that the upload really runs beside the steps
 };
 
@@ -281,6 +286,10 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   a->launches = 0;
   a->wslot = 0;
   a->host_pack2 = nullptr;
+  a->ids_host[0] = a->ids_host[1] = nullptr;
+  a->ids_copied[0] = a->ids_copied[1] = nullptr;
+  a->ids_in_flight[0] = a->ids_in_flight[1] = false;
+  a->ids_next = 0;
   a->copy_stream = nullptr;
   a->upload_done = a->image_free = nullptr;
   a->image_free_recorded = a->pending = false;
@@ -343,6 +352,10 @@ void marl_actor_destroy(marl_actor_t* a) {
     cudaEventDestroy(a->upload_done);
     cudaEventDestroy(a->image_free);
     cudaFreeHost(a->host_pack2);
+  }
+  for (int i = 0; i < 2; ++i) {
+    if (a->ids_host[i]) cudaFreeHost(a->ids_host[i]);
+    if (a->ids_copied[i]) cudaEventDestroy(a->ids_copied[i]);
   }
   if (a->own_ring) cudaFree(a->ring);
   if (a->own_state) cudaFree(a->state);
@@ -595,8 +608,22 @@ static int step_list(marl_actor* a, const int32_t* env_ids, int32_t M, const flo
     if (rcs) return rcs;
   }
   int32_t* d_ids = reinterpret_cast<int32_t*>(a->state + a->so.ids);
-  // pageable source: the copy has left the caller's array when the call returns
-  CU_TRY(cudaMemcpyAsync(d_ids, env_ids, sizeof(int32_t) * (size_t)M, cudaMemcpyHostToDevice, a->stream));
+  // The caller's array (pageable or pinned) is free again when this call returns: the validated list is copied into
+  // pinned staging owned by the actor and uploaded from there.  Two staging buffers take turns, each guarded by the
+  // event of its last upload, so filling one never overwrites a copy that is still in flight.
+  if (!a->ids_host[0]) {
+    for (int i = 0; i < 2; ++i) {
+      CU_TRY(cudaMallocHost(reinterpret_cast<void**>(&a->ids_host[i]), sizeof(int32_t) * (size_t)c.n_envs));
+      CU_TRY(cudaEventCreateWithFlags(&a->ids_copied[i], cudaEventDisableTiming));
+    }
+  }
+  const int ib = a->ids_next;
+  a->ids_next ^= 1;
+  if (a->ids_in_flight[ib]) CU_TRY(cudaEventSynchronize(a->ids_copied[ib]));
+  memcpy(a->ids_host[ib], env_ids, sizeof(int32_t) * (size_t)M);
+  CU_TRY(cudaMemcpyAsync(d_ids, a->ids_host[ib], sizeof(int32_t) * (size_t)M, cudaMemcpyHostToDevice, a->stream));
+  CU_TRY(cudaEventRecord(a->ids_copied[ib], a->stream));
+  a->ids_in_flight[ib] = true;
   ActorParams p;
   fill_params(a, p);
   p.T = 1;

@@ -9,16 +9,20 @@
 // array inside the library image instead of caller- or library-allocated memory.
 //
 // Consequences of the fixed array, all part of the contract:
-//   * its size is MARL_NOALLOC_SCRATCH_BYTES; every GPU whose context loads this library holds that much
-//     memory until the process exits, whether or not the entry point is ever called;
+//   * its size is MARL_NOALLOC_SCRATCH_BYTES.  CUDA loads the parts of a library image on first use, and this
+//     file holds nothing but the array, so the driver places the array on a GPU - and takes that much of its
+//     memory, until the process exits - when this entry point is first called with that GPU current.  That
+//     first call is the set-up call: make it at start-up, BEFORE the rest of the device memory goes to the
+//     caller's pool; a call with T = 0 does the set-up and nothing else.  Every later call on that device
+//     touches no allocator at all;
 //   * a configuration whose staging for ONE environment step does not fit is rejected with MARL_ENOMEM;
 //     larger T simply runs in more windows;
 //   * all actors and all calls on a device share the array.  It keeps whatever the previous call left in
 //     it; nothing in it has to start at zero, because every window is completely rewritten by the
 //     generator kernels before the actor kernel reads it.  Two calls whose GPU work overlaps (different
 //     streams, different host threads) race on it: serialise them;
-//   * the first call on a device looks up the array's device address (cudaGetSymbolAddress).  Make that
-//     first call outside any stream capture.
+//   * the set-up call looks up the array's device address (cudaGetSymbolAddress), which synchronises.  Make
+//     it outside any stream capture.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -57,6 +61,10 @@ uint8_t* scratch_on_current_device(cudaError_t* err) {
 
 extern "C" int marl_rollout_noalloc(marl_actor_t* a, const marl_synth_env_t* env, int32_t T, double eps_start,
                                     double eps_end, int32_t anneal_steps) {
+  if (T == 0) {  // set-up only: the driver places the array on the current device now
+    cudaError_t e0 = cudaSuccess;
+    return scratch_on_current_device(&e0) ? MARL_OK : MARL_ECUDA;
+  }
   if (!a || !env || T < 1) return MARL_EINVAL;
   marl_ring_view_t rv;
   int rc = marl_ring_view(a, &rv);

@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def guarded_buffers():
+    """Every Actor of the test-suite gets guard bytes around its ring, state and work buffers (the stand-in for a
+    memory checker); they are verified when the actor is destroyed."""
+    from paper_2205_05248_b200 import binding
+    old = binding.GUARD_BYTES
+    binding.GUARD_BYTES = 4096
+    yield
+    binding.GUARD_BYTES = old

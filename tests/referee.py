@@ -22,9 +22,12 @@ from paper_2205_05248_b200 import binding, workloads
 
 RTOL = {"fp32": 1e-5, "bf16": 2e-2}
 # Share of greedy decisions that may be near-ties.  fp32 path: the two sides differ by accumulation order
-# (about 1e-6 in Q).  bf16 path: operand roundings can flip and the kernel uses the hardware tanh
-# approximation, so Q differs by about 1e-3 and proportionally more decisions fall inside the tie band.
-NEAR_TIE_BUDGET = {"fp32": 1e-4, "bf16": 2e-3}
+# (about 1e-6 in Q).  bf16 path: operand roundings can flip and the tensor-core kernels use the hardware tanh
+# approximation, so Q differs by about 1e-3 and proportionally more decisions fall inside the tie band; the
+# rate is set from the rates measured at full size (listed with the results of each workload) with a margin
+# of about three.  A case with few rows may always have NEAR_TIE_FLOOR_ROWS of them.
+NEAR_TIE_BUDGET = {"fp32": 1e-4, "bf16": 4e-4}
+NEAR_TIE_FLOOR_ROWS = {"fp32": 0, "bf16": 2}
 
 
 def row_rel_err(got: np.ndarray, want: np.ndarray) -> np.ndarray:
@@ -52,16 +55,44 @@ def run_gpu_rollout(cfg, weights, kernel="auto", T=None, splits=None, want_q=Tru
     return actor, acts, q
 
 
+TRACES = ("avail", "q", "action_free", "explore", "slot", "pos")   # what the referee reads of the oracle's traces
+
+
+def near_tie_rows_allowed(precision, greedy_rows, budget=None, floor_rows=None):
+    """Near-ties a case may have: the budgeted share of its greedy decisions, at least the floor."""
+    budget = NEAR_TIE_BUDGET[precision] if budget is None else budget
+    floor_rows = NEAR_TIE_FLOOR_ROWS[precision] if floor_rows is None else floor_rows
+    return max(int(budget * greedy_rows), floor_rows if budget > 0 else 0)
+
+
+def check_near_ties(near, q_orc, q_gpu, a_orc, a_gpu, explore):
+    """Every row where the oracle's free choice differs from the library's: it must be a greedy row, and the two
+    actions' oracle Q values must be closer than the tie band plus twice that row's measured Q difference (each of
+    the two values moves by at most that much between the two sides).  near: [K][3] indices (t, x, i).
+    Returns the largest gap seen."""
+    if len(near) == 0:
+        return 0.0
+    t, x, i = near[:, 0], near[:, 1], near[:, 2]
+    assert not explore[t, x, i].any(), "an exploring row chose differently"
+    qo = q_orc[t, x, i].astype(np.float64)
+    qg = q_gpu[t, x, i].astype(np.float64)
+    rows = np.arange(len(near))
+    gap = np.abs(qo[rows, a_orc[t, x, i]] - qo[rows, a_gpu[t, x, i]])
+    bound = 1e-4 + 2.0 * np.max(np.abs(qo - qg), axis=-1)
+    worst = int(np.argmax(gap - bound))
+    assert (gap <= bound).all(), (f"actions differ at {tuple(near[worst])} with an oracle Q gap of {gap[worst]:.3e} "
+                                  f"(allowed {bound[worst]:.3e})")
+    return float(gap.max())
+
+
 def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_tie_budget=None, n_threads=None,
-            weight_schedule=()):
+            weight_schedule=(), near_tie_floor_rows=None):
     """Checks parts 1-4 for the listed environments (default: all).  Returns a summary dict.
     weight_schedule: (step, weights) pairs in rising step order; the oracle switches to that network at that step."""
     T = cfg["T"] if T is None else T
     E, n, A, H = cfg["E"], cfg["n"], cfg["A"], cfg["H"]
     ids = np.arange(E) if env_ids is None else np.asarray(env_ids)
     rtol = RTOL[cfg["precision"]]
-    if near_tie_budget is None:
-        near_tie_budget = NEAR_TIE_BUDGET[cfg["precision"]]
     tids = torch.as_tensor(ids, device=gpu_actions.device, dtype=torch.long)
     g_act = gpu_actions[:T].index_select(1, tids).cpu().numpy()
     g_q = gpu_q[:T].index_select(1, tids).cpu().numpy()
@@ -74,7 +105,7 @@ def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_
             sess.set_weights(weight_schedule[k - 1][1])
         if cuts[k + 1] > cuts[k]:
             parts.append(sess.rollout(cfg["env"], cuts[k + 1] - cuts[k], cfg["eps_start"], cfg["eps_end"],
-                                      cfg["anneal_steps"], adopt=g_act[cuts[k]:cuts[k + 1]]))
+                                      cfg["anneal_steps"], adopt=g_act[cuts[k]:cuts[k + 1]], trace=TRACES))
     tr = {key: np.concatenate([part[key] for part in parts]) for key in parts[0]}
 
     # ---- part 2: the GPU's decision follows from its own Q row ----
@@ -100,14 +131,9 @@ def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_
     # ---- part 4: near-ties ----
     greedy_rows = int((tr["explore"] == 0).sum())
     near = np.argwhere(tr["action_free"] != g_act)
-    for (t, x, i) in near[:64]:
-        assert tr["explore"][t, x, i] == 0
-        a_o, a_g = tr["action_free"][t, x, i], g_act[t, x, i]
-        gap = abs(float(tr["q"][t, x, i, a_o]) - float(tr["q"][t, x, i, a_g]))
-        scale = max(float(np.max(np.abs(tr["q"][t, x, i]))), 1e-3)
-        assert gap <= 1e-4 + 2 * rtol * scale, f"actions differ at {(t, x, i)} with an oracle Q gap of {gap:.3e}"
-    frac = len(near) / max(greedy_rows, 1)
-    assert frac <= near_tie_budget, f"{len(near)} near-ties in {greedy_rows} greedy decisions"
+    max_gap = check_near_ties(near, tr["q"], g_q, tr["action_free"], g_act, tr["explore"])
+    allowed = near_tie_rows_allowed(cfg["precision"], greedy_rows, near_tie_budget, near_tie_floor_rows)
+    assert len(near) <= allowed, f"{len(near)} near-ties in {greedy_rows} greedy decisions ({allowed} allowed)"
 
     # ---- part 1: integer state, ring and headers ----
     assert np.array_equal(st["last_action"].index_select(0, tids).cpu().numpy(), sess.last_action)
@@ -142,8 +168,28 @@ def referee(cfg, weights, actor, gpu_actions, gpu_q, env_ids=None, T=None, near_
         assert counters["agent_steps"] == oc[oracle.CNT_STEPS] and counters["episodes"] == oc[oracle.CNT_EPISODES]
         assert counters["explored"] == oc[oracle.CNT_EXPLORE] and counters["truncated"] == oc[oracle.CNT_TRUNCATED]
         assert counters["no_avail"] == oc[oracle.CNT_NO_AVAIL]
-    return dict(near_ties=len(near), greedy_rows=greedy_rows, q_err=float(q_err.max()), h_err=float(h_err.max()),
-                rows=N, episodes=int(sess.counters[oracle.CNT_EPISODES]), kernel=actor.kernel_name)
+    return dict(near_ties=len(near), greedy_rows=greedy_rows, near_tie_rate=len(near) / max(greedy_rows, 1),
+                near_tie_max_gap=max_gap, envs=len(ids), q_err=float(q_err.max()), h_err=float(h_err.max()), rows=N, episodes=int(sess.counters[oracle.CNT_EPISODES]), kernel=actor.kernel_name)
+
+
+def sample_env_tiles(E: int, tile_envs: int, count: int, grid: int = 148, seed: int = 0) -> np.ndarray:
+    """At least `count` environment ids made of whole tiles of `tile_envs` consecutive environments: the first and
+    the last tile, and seeded tiles spread evenly over the waves of a launch (a block of a `grid`-block launch
+    takes tiles b, b + grid, b + 2 grid, ...; wave w holds tiles [w grid, (w + 1) grid))."""
+    if count >= E:
+        return np.arange(E)
+    tiles = (E + tile_envs - 1) // tile_envs
+    want = min(tiles, (count + tile_envs - 1) // tile_envs)
+    waves = (tiles + grid - 1) // grid
+    rng = np.random.default_rng(seed)
+    chosen = {0, tiles - 1}
+    w = 0
+    while len(chosen) < want:                       # round-robin over the waves
+        lo, hi = w * grid, min((w + 1) * grid, tiles)
+        chosen.add(int(rng.integers(lo, hi)))
+        w = (w + 1) % waves
+    ids = np.concatenate([np.arange(t * tile_envs, min((t + 1) * tile_envs, E)) for t in sorted(chosen)])
+    return ids
 
 
 def sample_envs(E: int, count: int, seed: int = 0) -> np.ndarray:

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_2205_05248_b200 import binding, workloads
-from referee import referee, run_gpu_rollout, sample_envs
+from referee import referee, run_gpu_rollout, sample_env_tiles
 from test_gpu_parity import _assert_same_rollout
 
 pytestmark = pytest.mark.gpu
@@ -48,9 +48,8 @@ def test_published_weights_take_effect_at_their_step(kernel, prec, shape):
         _assert_same_rollout(actor, acts, q, ref, acts_r, q_r)
     # and against the oracle, which switches networks at the same step
     actor, acts, q = runs[0]
-    ids = sample_envs(cfg["E"], 40, seed=3)
-    res = referee(cfg, w0, actor, acts, q, env_ids=ids, near_tie_budget=2e-3, weight_schedule=[(switch, w1)])
-    assert res["rows"] == cfg["T"] * len(ids) * cfg["n"]
+    res = referee(cfg, w0, actor, acts, q, weight_schedule=[(switch, w1)])       # every environment
+    assert res["rows"] == cfg["T"] * cfg["E"] * cfg["n"]
     # the new network matters: a rollout that never switches differs after the switch step
     same, acts_s, q_s = run_gpu_rollout(cfg, w0, kernel=kernel)
     assert torch.equal(q_s[:switch], q[:switch]) and not torch.allclose(q_s[switch:], q[switch:], rtol=1e-2, atol=1e-3)
@@ -92,8 +91,8 @@ def test_publication_rules():
 
 def test_published_weights_full_size_bench_configuration():
     """The configuration `bench.py --refresh` times: workload 5 at full size, one staged 64-step rollout with a
-    publication that takes effect 32 steps in (two launches of 32 steps); the oracle recomputes sampled environments
-    with the same switch."""
+    publication that takes effect 32 steps in (two launches of 32 steps); the oracle recomputes 4096 environments
+    (whole tiles) with the same switch."""
     cfg = workloads.config(5)
     T = cfg["T"]
     w0 = workloads.make_weights(cfg)
@@ -108,7 +107,9 @@ def test_published_weights_full_size_bench_configuration():
     actor.rollout_staged(*staged, T, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
     torch.cuda.synchronize()
     assert actor.launch_count - launches == 2 and actor.weights_version == 2
-    res = referee(cfg, w0, actor, acts, q, env_ids=sample_envs(cfg["E"], 24, seed=6), weight_schedule=[(T // 2, w1)])
+    ids = sample_env_tiles(cfg["E"], 128 // cfg["n"], 4096, seed=6)      # whole tiles from every wave of both launches
+    res = referee(cfg, w0, actor, acts, q, env_ids=ids, weight_schedule=[(T // 2, w1)])
+    assert res["envs"] >= 4096
     print(f"cfg5 full size with a publication: {res}")
     status, counters = actor.status()
     assert status == 0 and counters["agent_steps"] == cfg["E"] * cfg["n"] * T
