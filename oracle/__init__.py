@@ -36,7 +36,8 @@ def build(force: bool = False) -> str:
 class Dims(C.Structure):
     _fields_ = [("n_envs", C.c_int32), ("n_agents", C.c_int32), ("obs_dim", C.c_int32),
                 ("n_actions", C.c_int32), ("hidden", C.c_int32), ("ring_episodes", C.c_int32),
-                ("ring_steps", C.c_int32), ("precision", C.c_int32), ("seed", C.c_uint64)]
+                ("ring_steps", C.c_int32), ("precision", C.c_int32), ("seed", C.c_uint64),
+                ("n_types", C.c_int32), ("reserved", C.c_int32), ("agent_type", C.c_void_p)]
 
 
 class Env(C.Structure):
@@ -95,11 +96,20 @@ def _c(a, dtype):
 
 
 def make_dims(cfg: dict) -> Dims:
-    """cfg uses the keys E, n, D, A, H, C, L, precision ('fp32'|'bf16' or 0|1), seed."""
+    """cfg uses the keys E, n, D, A, H, C, L, precision ('fp32'|'bf16' or 0|1), seed, and optionally agent_type
+    (a list of n unit types: with more than one type the weights are a list of networks, one per type)."""
     prec = cfg["precision"]
     prec = {"fp32": 0, "bf16": 1}.get(prec, prec)
-    return Dims(cfg["E"], cfg["n"], cfg["D"], cfg["A"], cfg["H"], cfg["C"], cfg["L"], int(prec),
-                int(cfg["seed"]))
+    d = Dims(cfg["E"], cfg["n"], cfg["D"], cfg["A"], cfg["H"], cfg["C"], cfg["L"], int(prec), int(cfg["seed"]),
+             0, 0, None)
+    types = cfg.get("agent_type")
+    if types is not None:
+        arr = np.ascontiguousarray(types, dtype=np.int32)
+        assert arr.shape == (cfg["n"],) and arr.min() >= 0
+        d._keep_types = arr                      # keeps the array alive as long as the struct
+        d.n_types = int(arr.max()) + 1
+        d.agent_type = arr.ctypes.data_as(C.c_void_p)
+    return d
 
 
 def make_env(env: dict) -> Env:
@@ -132,9 +142,17 @@ def hardware_threads() -> int:
     return int(lib().oracle_hardware_threads())
 
 
-def _weights_struct(w: dict):
-    keep = {k: _c(w[k], np.float32) for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")}
-    return _Weights(*[_ptr(keep[k]) for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")]), keep
+_WNAMES = ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")
+
+
+def _weights_struct(w):
+    """One network (a dict) or, for per-type networks, a list of them (an array of structs on the C side)."""
+    if isinstance(w, dict):
+        keep = {k: _c(w[k], np.float32) for k in _WNAMES}
+        return _Weights(*[_ptr(keep[k]) for k in _WNAMES]), keep
+    keep = [{k: _c(wk[k], np.float32) for k in _WNAMES} for wk in w]
+    arr = (_Weights * len(keep))(*[_Weights(*[_ptr(kk[k]) for k in _WNAMES]) for kk in keep])
+    return arr, keep
 
 
 def env_emit(cfg: dict, env: dict, t: int, e: int):

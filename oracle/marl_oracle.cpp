@@ -127,6 +127,13 @@ struct oracle_dims {
   int32_t ring_steps;     // L
   int32_t precision;      // 0 = fp32, 1 = bf16 weights and operands
   uint64_t seed;          // key of the epsilon stream
+  // Heterogeneous teams (Table I lists a scenario whose team mixes two unit types; Sec. IV discusses it): each
+  // unit type may have a network of its own instead of the one shared network.  n_types <= 1 or a null
+  // agent_type: one network for every agent.  Otherwise agent i is decided for by network agent_type[i], and
+  // every routine below that takes `const oracle_weights* w` is given an array of n_types networks.
+  int32_t n_types;
+  int32_t reserved;
+  const int32_t* agent_type;  // [n], each in [0, n_types)
 };
 
 // Seeded synthetic environment standing in for the simulator of Algorithm 1 (Env.step / Env.done).
@@ -401,6 +408,12 @@ void oracle_init(const oracle_dims* d, const int32_t* env_ids, int32_t Es, oracl
 //       with another implementation across numerical near-ties); the own choice is still traced.
 //   tr / tstep: optional trace, written at step index tstep of a trace holding Es rows per step.
 // ---------------------------------------------------------------------------------------------------
+// The network that decides for agent i: the shared one, or the one of the agent's unit type.
+static const oracle_weights* network_of(const oracle_dims* d, const oracle_weights* w, int agent) {
+  if (d->n_types <= 1 || d->agent_type == nullptr) return w;
+  return w + d->agent_type[agent];
+}
+
 static void step_range(const oracle_dims* d, const oracle_weights* w, const int32_t* env_ids, int x0,
                        int x1, int32_t Es, uint32_t t, float eps, const float* obs,
                        const uint8_t* avail, const float* reward, const uint8_t* done,
@@ -425,7 +438,8 @@ static void step_range(const oracle_dims* d, const oracle_weights* w, const int3
       const float* o = obs + row * D;
       const uint8_t* av = avail + row * A;
       float* hp = st->h + row * H;
-      oracle_agent_forward(d, w, o, i, st->last_action[row], hp, q.data(), hnew.data() + (size_t)i * H);
+      oracle_agent_forward(d, network_of(d, w, i), o, i, st->last_action[row], hp, q.data(),
+                           hnew.data() + (size_t)i * H);
       uint8_t ex = 0, na = 0;
       float u = 0.f;
       const int32_t a_free = oracle_select_action(q.data(), av, A, eps, d->seed, t, (uint32_t)e,
@@ -578,7 +592,7 @@ void oracle_step_lagged(const oracle_dims* d, const oracle_weights* w, const int
       const size_t row = (size_t)x * n + i;
       const float* o = obs + row * D;
       const uint8_t* av = avail + row * A;
-      oracle_agent_forward(d, w, o, i, st->last_action[row], st->h + row * H, q.data(),
+      oracle_agent_forward(d, network_of(d, w, i), o, i, st->last_action[row], st->h + row * H, q.data(),
                            hnew.data() + (size_t)i * H);
       uint8_t ex = 0, na = 0;
       float u = 0.f;

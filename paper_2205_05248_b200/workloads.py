@@ -104,3 +104,23 @@ def make_weights(cfg: dict, seed: int | None = None, bias_scale: float = 1.0) ->
 
     return dict(W1=xavier(H, I), b1=bias(H, I), W_ih=xavier(3 * H, H), b_ih=bias(3 * H, H),
                 W_hh=xavier(3 * H, H), b_hh=bias(3 * H, H), W2=xavier(A, H), b2=bias(A, H))
+
+
+def typed(cfg: dict, agent_type=None) -> dict:
+    """The same workload with one network per unit type: ``agent_type`` lists every agent's type (default: the two
+    types of the workload's typed feature blocks - agents [0, n_type0) type 0, the others type 1)."""
+    c = dict(cfg)
+    if agent_type is None:
+        n0 = cfg["env"]["n_type0"]
+        assert 0 < n0 < cfg["n"], "the workload has no unit types of its own: pass agent_type"
+        agent_type = [0] * n0 + [1] * (cfg["n"] - n0)
+    assert len(agent_type) == cfg["n"] and sorted(set(agent_type)) == list(range(max(agent_type) + 1))
+    c["agent_type"] = [int(t) for t in agent_type]
+    c["name"] = cfg.get("name", "cfg") + "_typed"
+    return c
+
+
+def make_weights_typed(cfg: dict, seed: int | None = None) -> list:
+    """One network per unit type of ``typed(cfg)``, each drawn like ``make_weights`` from a seed of its own."""
+    base = cfg["seed"] if seed is None else seed
+    return [make_weights(cfg, seed=base + 7919 * (k + 1)) for k in range(max(cfg["agent_type"]) + 1)]
