@@ -51,8 +51,8 @@ extern "C" {
 #define MARL_PRECISION_FP32 0 /* fp32 weights, fp32 FFMA arithmetic */
 #define MARL_PRECISION_BF16 1 /* weight matrices and matmul operands rounded to bf16 (RNE), fp32 accumulate */
 
-#define MARL_KERNEL_AUTO 0   /* a tensor-core kernel (the pipelined one where the shape allows it) where supported and
-                              * the batch is large, else FFMA */
+#define MARL_KERNEL_AUTO 0   /* bf16: a tensor-core kernel (the pipelined one where the shape allows it) wherever the
+                              * shape is supported, at every batch size; otherwise, and for fp32, FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
 #define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, n_agents * n_actions
@@ -61,6 +61,8 @@ extern "C" {
                                         * not a 16-byte multiple, an environment count that is not a multiple of 4)
                                         * fall back, per call, to the one-tile kernel where the shape allows it,
                                         * else to the FFMA kernel */
+
+#define MARL_MAX_AGENT_TYPES 4
 
 #define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
 #define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
@@ -81,7 +83,8 @@ typedef struct {
   int32_t ring_steps;    /* L: steps per slot; an episode reaching L steps is truncated */
   int32_t precision;     /* MARL_PRECISION_* */
   int32_t kernel;        /* MARL_KERNEL_* */
-  int32_t reserved;      /* must be 0 */
+  int32_t n_agent_types; /* 0 or 1: one network shared by all agents; 2..MARL_MAX_AGENT_TYPES: room for that many
+                          * per-type networks (marl_actor_set_weights_typed) */
   uint64_t seed;         /* Philox key of the exploration stream */
   void* stream;          /* cudaStream_t, borrowed; NULL = the legacy default stream */
   /* Device memory.  NULL = the library allocates with cudaMalloc and owns it.  Otherwise the caller's
@@ -181,6 +184,20 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out);
 int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, const float* W_ih,
                            const float* b_ih, const float* W_hh, const float* b_hh, const float* W2,
                            const float* b2, uint64_t version);
+
+/* One network per unit type, for heterogeneous teams (Table I of the paper lists a scenario whose team mixes two
+ * unit types, and Sec. IV discusses it; the paper's agents share one network, so this is an extension of the
+ * worker's decision step of Algorithm 2, not something the paper prints).  Agent i of every environment is decided
+ * for by network agent_type[i]; the network input keeps its agent-id one-hot.  HOST arrays: agent_type i32[n], each
+ * in [0, n_types); the eight weight arrays as for marl_actor_set_weights with a leading [n_types] axis
+ * (W1 [K][H][D+n+A], b1 [K][H], ...).  n_types must not exceed the n_agent_types the actor was created with.
+ * Blocking, like marl_actor_set_weights, and a pending publication is dropped.  With n_types > 1 the steps run on
+ * the CUDA-core kernel (both precisions; the products are evaluated once per type), marl_actor_publish_weights is
+ * refused, and marl_actor_kernel_name reports "ffma"; a later marl_actor_set_weights returns to the shared network
+ * and the kernel chosen at creation. */
+int marl_actor_set_weights_typed(marl_actor_t* a, int32_t n_types, const int32_t* agent_type, const float* W1,
+                                 const float* b1, const float* W_ih, const float* b_ih, const float* W_hh,
+                                 const float* b_hh, const float* W2, const float* b2, uint64_t version);
 
 /* The learner's refresh of the shared model while the workers run (Sec. III-B: the learner updates the model in
  * the shared memory pool; Algorithm 2: a worker gets the parameters at the start of an iteration).  The network

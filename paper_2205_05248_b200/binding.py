@@ -28,7 +28,8 @@ GUARD_BYTES = 0
 GUARD_PATTERN = 0xA5
 
 EXPORTS = [
-    "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_publish_weights",
+    "marl_actor_query_sizes", "marl_actor_create", "marl_actor_set_weights", "marl_actor_set_weights_typed",
+    "marl_actor_publish_weights",
     "marl_actor_weights_version",
     "marl_actor_step", "marl_actor_step_subset", "marl_actor_step_lagged", "marl_actor_step_host", "marl_env_generate", "marl_rollout_staged", "marl_rollout",
     "marl_actor_set_trace", "marl_ring_view", "marl_ring_sample", "marl_actor_get_state", "marl_actor_set_state",
@@ -45,7 +46,7 @@ class MarlError(RuntimeError):
 class Config(C.Structure):
     _fields_ = [("n_envs", C.c_int32), ("n_agents", C.c_int32), ("obs_dim", C.c_int32), ("n_actions", C.c_int32),
                 ("hidden", C.c_int32), ("ring_episodes", C.c_int32), ("ring_steps", C.c_int32),
-                ("precision", C.c_int32), ("kernel", C.c_int32), ("reserved", C.c_int32), ("seed", C.c_uint64),
+                ("precision", C.c_int32), ("kernel", C.c_int32), ("n_agent_types", C.c_int32), ("seed", C.c_uint64),
                 ("stream", C.c_void_p), ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
                 ("state_mem", C.c_void_p), ("state_bytes", C.c_size_t), ("work_mem", C.c_void_p),
                 ("work_bytes", C.c_size_t)]
@@ -109,6 +110,7 @@ def load_library():
         lib.marl_actor_query_sizes.argtypes = [C.POINTER(Config), C.POINTER(Sizes)]
         lib.marl_actor_create.argtypes = [C.POINTER(Config), C.POINTER(P)]
         lib.marl_actor_set_weights.argtypes = [P] + [P] * 8 + [C.c_uint64]
+        lib.marl_actor_set_weights_typed.argtypes = [P, C.c_int32, P] + [P] * 8 + [C.c_uint64]
         lib.marl_actor_publish_weights.argtypes = [P] + [P] * 8 + [C.c_uint64, C.c_uint64]
         lib.marl_actor_step.argtypes = [P, P, P, P, P, C.c_float, P]
         lib.marl_actor_step_host.argtypes = [P, P, P, P, P, C.c_float, P]
@@ -149,6 +151,7 @@ def make_config(cfg: dict, kernel: str = "auto") -> Config:
     c.n_envs, c.n_agents, c.obs_dim, c.n_actions, c.hidden = cfg["E"], cfg["n"], cfg["D"], cfg["A"], cfg["H"]
     c.ring_episodes, c.ring_steps, c.precision, c.kernel = cfg["C"], cfg["L"], int(prec), KERNEL[kernel]
     c.seed = int(cfg["seed"])
+    c.n_agent_types = (max(cfg["agent_type"]) + 1) if cfg.get("agent_type") is not None else 0
     return c
 
 
@@ -256,6 +259,16 @@ class Actor:
                 for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")]
         _check(self.lib.marl_actor_set_weights(self.handle, *[a.ctypes.data_as(C.c_void_p) for a in arrs],
                                                C.c_uint64(version)))
+
+    def set_weights_typed(self, ws: list, agent_type=None, version: int = 1):
+        """marl_actor_set_weights_typed: one network (a dict like ``set_weights`` takes) per unit type; agent_type
+        defaults to the configuration's."""
+        import numpy as np
+        types = np.ascontiguousarray(self.cfg["agent_type"] if agent_type is None else agent_type, dtype=np.int32)
+        arrs = [np.ascontiguousarray(np.stack([w[k] for w in ws]), dtype=np.float32)
+                for k in ("W1", "b1", "W_ih", "b_ih", "W_hh", "b_hh", "W2", "b2")]
+        _check(self.lib.marl_actor_set_weights_typed(self.handle, C.c_int32(len(ws)), types.ctypes.data_as(C.c_void_p),
+                                                     *[a.ctypes.data_as(C.c_void_p) for a in arrs], C.c_uint64(version)))
 
     def publish_weights(self, w: dict, version: int, effective_step: int):
         """marl_actor_publish_weights: the network in use from global step effective_step on."""
@@ -373,8 +386,11 @@ class Actor:
         i32 = u8[: u8.numel() // 4 * 4].view(torch.int32)
         ss, ps = v.slot_stride, v.step_stride
 
+        # (as_strided offsets count from the start of the storage, and ring_mem may itself start inside one)
+        so4, so1 = f32.storage_offset(), u8.storage_offset()
+
         def f(off, shape_tail, stride_tail):
-            return torch.as_strided(f32, (Cn, L, *shape_tail), (ss // 4, ps // 4, *stride_tail), (base_off + off) // 4)
+            return torch.as_strided(f32, (Cn, L, *shape_tail), (ss // 4, ps // 4, *stride_tail), so4 + (base_off + off) // 4)
 
         def hdr(ptr, dtype, count):
             o = ptr - u8.data_ptr()
@@ -383,9 +399,9 @@ class Actor:
 
         out = dict(
             obs=f(v.off_obs, (n, D), (D, 1)), q=f(v.off_q, (n, A), (A, 1)), reward=f(v.off_reward, (), ()),
-            action=torch.as_strided(i32, (Cn, L, n), (ss // 4, ps // 4, 1), (base_off + v.off_action) // 4),
-            avail=torch.as_strided(u8, (Cn, L, n, A), (ss, ps, A, 1), base_off + v.off_avail),
-            done=torch.as_strided(u8, (Cn, L), (ss, ps), base_off + v.off_done),
+            action=torch.as_strided(i32, (Cn, L, n), (ss // 4, ps // 4, 1), so4 + (base_off + v.off_action) // 4),
+            avail=torch.as_strided(u8, (Cn, L, n, A), (ss, ps, A, 1), so1 + base_off + v.off_avail),
+            done=torch.as_strided(u8, (Cn, L), (ss, ps), so1 + base_off + v.off_done),
             slot_epid=hdr(v.slot_epid, torch.int64, Cn), slot_len=hdr(v.slot_len, torch.int32, Cn),
             slot_complete=hdr(v.slot_complete, torch.uint8, Cn))
         out["meta"] = {k: getattr(v, k) for k, _ in RingView._fields_}

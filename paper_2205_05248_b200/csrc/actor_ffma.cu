@@ -88,7 +88,13 @@ __device__ __forceinline__ float4 round4(float4 v, bool lowp) {
   return v;
 }
 
-template <bool WS>
+// TYPED: one network per unit type (heterogeneous teams).  The tile's rows mix types, and a thread's register tile
+// shares each weight value among its four rows, so the three products run once per type on that type's image with
+// the operand of every row of another type replaced by zero: fma(0, w, acc) leaves acc as it is, so a row
+// accumulates exactly the products of its own network.  Biases, the one-hot columns and fc2 (one row per thread)
+// read the row's own image directly.  The images are read through the read-only path (they do not fit shared memory
+// together).
+template <bool WS, bool TYPED>
 __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_constant__ ActorParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
   const FfmaSmem sl = ffma_smem_layout(p.n, p.D, p.A, p.H);
@@ -105,6 +111,12 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   const bool lowp = p.prec == MARL_PRECISION_BF16;
   const int hbuf = FF_RMAX * Hp;  // floats per hidden buffer
   const int tx = tid & 15, ty = tid >> 4;
+  const int ntypes = TYPED ? p.n_types : 1;
+  const size_t tstride = TYPED ? p.type_stride : 0;
+  auto row_type = [&](int r) -> int { return TYPED ? (int)((p.agent_type_bits >> (2 * (r % n))) & 3ull) : 0; };
+  int rt[4];  // unit type of this thread's four rows
+#pragma unroll
+  for (int m = 0; m < 4; ++m) rt[m] = row_type(ty + 16 * m);
 
   unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
   uint32_t st_bits = 0;
@@ -268,19 +280,23 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       for (int jb = 0; jb < H; jb += 64) {
         const int j0 = jb + tx * 4;
         float acc[4][4];
-        {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(p.b1 + j0));
 #pragma unroll
-          for (int m = 0; m < 4; ++m) { acc[m][0] = b.x; acc[m][1] = b.y; acc[m][2] = b.z; acc[m][3] = b.w; }
+        for (int m = 0; m < 4; ++m) {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(p.b1 + rt[m] * tstride + j0));
+          acc[m][0] = b.x; acc[m][1] = b.y; acc[m][2] = b.z; acc[m][3] = b.w;
         }
         const int K4 = (D + 3) & ~3;
+        for (int typ = 0; typ < ntypes; ++typ)
         for (int k = 0; k < K4; k += 4) {
           float4 xv[4];
 #pragma unroll
-          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xs + (ty + 16 * m) * Dp + k);
+          for (int m = 0; m < 4; ++m) {
+            xv[m] = *reinterpret_cast<const float4*>(xs + (ty + 16 * m) * Dp + k);
+            if (TYPED && rt[m] != typ) xv[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            const float4 w = wload4<WS>(W1T + (size_t)(k + kk) * H + j0);
+            const float4 w = wload4<WS>(W1T + typ * tstride + (size_t)(k + kk) * H + j0);
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
               const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
@@ -295,11 +311,11 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         for (int m = 0; m < 4; ++m) {
           const int r = ty + 16 * m;
           const int ai = r % n;
-          const float4 wid = wload4<WS>(W1T + (size_t)(D + ai) * H + j0);
+          const float4 wid = wload4<WS>(W1T + rt[m] * tstride + (size_t)(D + ai) * H + j0);
           float4 o = make_float4(acc[m][0] + wid.x, acc[m][1] + wid.y, acc[m][2] + wid.z, acc[m][3] + wid.w);
           const int last = la[r];
           if (last >= 0) {
-            const float4 wl = wload4<WS>(W1T + (size_t)(D + n + last) * H + j0);
+            const float4 wl = wload4<WS>(W1T + rt[m] * tstride + (size_t)(D + n + last) * H + j0);
             o.x += wl.x; o.y += wl.y; o.z += wl.z; o.w += wl.w;
           }
           o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
@@ -313,15 +329,17 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       for (int jb = 0; jb < H; jb += 64) {
         const int j0 = jb + tx * 4;
         float ar[4][4], az[4][4], ai_[4][4], ah[4][4];
-        {
-          const float4 bir = __ldg(reinterpret_cast<const float4*>(p.bih + j0));
-          const float4 biz = __ldg(reinterpret_cast<const float4*>(p.bih + H + j0));
-          const float4 bin = __ldg(reinterpret_cast<const float4*>(p.bih + 2 * H + j0));
-          const float4 bhr = __ldg(reinterpret_cast<const float4*>(p.bhh + j0));
-          const float4 bhz = __ldg(reinterpret_cast<const float4*>(p.bhh + H + j0));
-          const float4 bhn = __ldg(reinterpret_cast<const float4*>(p.bhh + 2 * H + j0));
 #pragma unroll
-          for (int m = 0; m < 4; ++m) {
+        for (int m = 0; m < 4; ++m) {
+          const float* bih = p.bih + rt[m] * tstride;
+          const float* bhh = p.bhh + rt[m] * tstride;
+          const float4 bir = __ldg(reinterpret_cast<const float4*>(bih + j0));
+          const float4 biz = __ldg(reinterpret_cast<const float4*>(bih + H + j0));
+          const float4 bin = __ldg(reinterpret_cast<const float4*>(bih + 2 * H + j0));
+          const float4 bhr = __ldg(reinterpret_cast<const float4*>(bhh + j0));
+          const float4 bhz = __ldg(reinterpret_cast<const float4*>(bhh + H + j0));
+          const float4 bhn = __ldg(reinterpret_cast<const float4*>(bhh + 2 * H + j0));
+          {
             ar[m][0] = bir.x + bhr.x; ar[m][1] = bir.y + bhr.y; ar[m][2] = bir.z + bhr.z; ar[m][3] = bir.w + bhr.w;
             az[m][0] = biz.x + bhz.x; az[m][1] = biz.y + bhz.y; az[m][2] = biz.z + bhz.z; az[m][3] = biz.w + bhz.w;
             ai_[m][0] = bin.x; ai_[m][1] = bin.y; ai_[m][2] = bin.z; ai_[m][3] = bin.w;
@@ -329,14 +347,18 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           }
         }
 #pragma unroll 1
-        for (int pass = 0; pass < 2; ++pass) {
+        for (int tp = 0; tp < 2 * ntypes; ++tp) {
+          const int pass = tp & 1, typ = tp >> 1;
           const float* act = pass == 0 ? ys : (hs + cur * hbuf);
-          const float* WT = pass == 0 ? WihT : WhhT;
+          const float* WT = (pass == 0 ? WihT : WhhT) + typ * tstride;
           const bool rnd = lowp && pass == 1;  // the hidden state is stored in fp32; its operand copy is rounded here
           for (int k = 0; k < H; k += 4) {
             float4 v[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) v[m] = round4(*reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k), rnd);
+            for (int m = 0; m < 4; ++m) {
+              v[m] = round4(*reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k), rnd);
+              if (TYPED && rt[m] != typ) v[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
               const float* wrow = WT + (size_t)(k + kk) * H3 + j0;
@@ -382,11 +404,12 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       // ---- phase D: fc2 (four threads per row, actions striped over them) ----
       {
         const int r = tid >> 2, part = tid & 3;
+        const size_t toff = row_type(r) * tstride;  // this row's own network
         float acc[8];
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
           const int a = part + 4 * m;
-          acc[m] = a < A ? __ldg(p.b2 + a) : 0.f;
+          acc[m] = a < A ? __ldg(p.b2 + toff + a) : 0.f;
         }
         const float* hv = hs + nxt * hbuf + r * Hp;
         for (int k = 0; k < H; k += 4) {
@@ -395,7 +418,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           for (int m = 0; m < 8; ++m) {
             const int a = part + 4 * m;
             if (a < A) {
-              const float4 w = wload4<WS>(W2 + (size_t)a * H + k);
+              const float4 w = wload4<WS>(W2 + toff + (size_t)a * H + k);
               acc[m] = fmaf(v.x, w.x, acc[m]);
               acc[m] = fmaf(v.y, w.y, acc[m]);
               acc[m] = fmaf(v.z, w.z, acc[m]);
@@ -518,15 +541,18 @@ size_t ffma_smem_bytes(int n, int D, int A, int H) { return ffma_smem_layout(n, 
 // Returns the number of kernels launched or a negative cudaError.
 int launch_actor_ffma(const ActorParams& p, int sms, cudaStream_t stream) {
   const FfmaSmem sl = ffma_smem_layout(p.n, p.D, p.A, p.H);
-  auto kernel = sl.wsmem ? actor_ffma_kernel<true> : actor_ffma_kernel<false>;
-  static uint32_t configured[2][SMEM_OPTIN_DEVICES];
+  const bool typed = p.n_types > 1;
+  const bool ws = sl.wsmem && !typed;
+  auto kernel = typed ? actor_ffma_kernel<false, true> : (ws ? actor_ffma_kernel<true, false> : actor_ffma_kernel<false, false>);
+  const size_t smem_bytes = ws ? sl.total : sl.off_w;
+  static uint32_t configured[3][SMEM_OPTIN_DEVICES];
   {
-    const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (uint32_t)sl.total, configured[sl.wsmem ? 1 : 0]);
+    const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (uint32_t)smem_bytes, configured[typed ? 2 : (ws ? 1 : 0)]);
     if (e != cudaSuccess) return -(int)e;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (grid < 1) grid = 1;
-  kernel<<<grid, FF_THREADS, sl.total, stream>>>(p);
+  kernel<<<grid, FF_THREADS, smem_bytes, stream>>>(p);
   const cudaError_t err = cudaGetLastError();
   return err == cudaSuccess ? 1 : -(int)err;
 }

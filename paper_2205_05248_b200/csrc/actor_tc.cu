@@ -107,6 +107,9 @@ void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b
     for (int j = 0; j < H; ++j) tla[a * TC_TAB + j] = bf16_value(W1[(size_t)j * I + D + n + a]);
 }
 
+// Environments per tile: as many as fit 128 rows.  (Spreading a batch of fewer tiles than SMs over partly filled
+// tiles was measured and gains nothing: a launch of T steps takes T times the per-step dependency chain of one
+// tile however few rows the tile holds.)
 void tc_tiling(int E, int n, int /*sms*/, int* ept, int* num_tiles) {
   *ept = TC_ROWS / n;
   *num_tiles = (E + *ept - 1) / *ept;

@@ -69,6 +69,11 @@ struct ActorParams {
   int32_t M;
   // T == 1 over a list: reward/done are the outcome of each environment's PREVIOUS action (committed at pos - 1)
   int32_t lagged;
+  // One network per unit type (FFMA kernel only): n_types > 1, the FFMA image of type k starts type_stride floats
+  // after the one of type k - 1, and agent i's type is bits 2i, 2i+1 of agent_type_bits.
+  int32_t n_types;
+  uint32_t type_stride;
+  uint64_t agent_type_bits;
 };
 
 // Everything the episode sampler needs (ring_sample.cu).  Passed by value.

@@ -110,8 +110,9 @@ static StateOffsets state_offsets(const marl_actor_config_t& c) {
   s.ep_count = cv.take(sizeof(int64_t) * c.n_envs);
   s.counters = cv.take(sizeof(uint64_t) * CNT_N);
   s.status = cv.take(sizeof(uint32_t) * 4);
+  const size_t types = c.n_agent_types > 1 ? (size_t)c.n_agent_types : 1;  // FFMA images of a typed actor, one per type
   for (int i = 0; i < 2; ++i) {
-    s.wff[i] = cv.take(ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
+    s.wff[i] = cv.take(types * ffma_weight_offsets(c.n_agents, c.obs_dim, c.n_actions, c.hidden).total);
     s.wpack[i] = cv.take(tc_wpack_bytes(c.n_agents, c.obs_dim, c.n_actions, c.hidden));
   }
   s.ids = cv.take(sizeof(int32_t) * (size_t)c.n_envs);  // environment list of a partial step
@@ -158,7 +159,8 @@ static int check_config(const marl_actor_config_t* c) {
   if (c->precision != MARL_PRECISION_FP32 && c->precision != MARL_PRECISION_BF16)
     return fail(MARL_EINVAL, "unknown precision");
   if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR_PIPELINED) return fail(MARL_EINVAL, "unknown kernel");
-  if (c->reserved != 0) return fail(MARL_EINVAL, "reserved must be 0");
+  if (c->n_agent_types < 0 || c->n_agent_types > MARL_MAX_AGENT_TYPES)
+    return fail(MARL_EINVAL, "n_agent_types must be in [0, %d]", MARL_MAX_AGENT_TYPES);
   if ((double)c->n_envs * c->n_agents > 1.0e9) return fail(MARL_EINVAL, "n_envs * n_agents too large");
   return MARL_OK;
 }
@@ -169,6 +171,9 @@ struct marl_actor {
   int device, sms;
   bool use_tc;   // a tensor-core kernel steps this actor
   bool use_tcp;  // ... the pipelined one (falls back to the one-tile kernel for inputs it cannot bulk-copy)
+  bool tc_allowed, tcp_allowed;  // the choice made at creation; per-type networks switch the tensor-core kernels off
+  int32_t n_types;               // > 1: per-type networks are loaded
+  uint64_t agent_type_bits;
   uint8_t *ring, *state, *work;
   bool own_ring, own_state, own_work;
   size_t work_bytes;
@@ -301,11 +306,17 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
     delete a;
     return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
   }
-  // Below a couple of 128-row tiles the FFMA kernel, which spreads 64-row tiles over more SMs, is used.
-  const bool big = (long long)cfg->n_envs * cfg->n_agents >= 256;
-  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED || (cfg->kernel == MARL_KERNEL_AUTO && big && tcp_ok);
-  a->use_tc = tc_ok && (cfg->kernel == MARL_KERNEL_TENSOR || cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED ||
-                        (cfg->kernel == MARL_KERNEL_AUTO && big));
+  // Kernel choice.  fp32 precision: the CUDA-core kernel (tensor cores cannot meet its 1e-5 tolerance).  bf16: a
+  // tensor-core kernel wherever the shape is supported, at every batch size - timed on the same rollouts from 24
+  // rows to 16384 (`bench.py --crossover`, table in the benchmark spec), one 128-row tcgen05 tile takes 3.4-4.6 us per
+  // environment step against 25-29 us for the CUDA-core kernel's 64-row tiles, so there is no batch size at which
+  // the CUDA cores win.
+  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED || (cfg->kernel == MARL_KERNEL_AUTO && tcp_ok);
+  a->use_tc = tc_ok && cfg->kernel != MARL_KERNEL_FFMA;
+  a->tcp_allowed = a->use_tcp;
+  a->tc_allowed = a->use_tc;
+  a->n_types = 1;
+  a->agent_type_bits = 0;
 
   auto bind = [&](void* mem, size_t have, size_t need, uint8_t** dst, bool* own, const char* what) -> int {
     if (mem) {
@@ -430,6 +441,58 @@ int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, co
   CU_TRY(cudaStreamSynchronize(a->stream));
   a->weights_version = version;
   a->have_weights = true;
+  a->n_types = 1;  // one shared network again: the kernels chosen at creation
+  a->agent_type_bits = 0;
+  a->use_tc = a->tc_allowed;
+  a->use_tcp = a->tcp_allowed;
+  return MARL_OK;
+}
+
+int marl_actor_set_weights_typed(marl_actor_t* a, int32_t n_types, const int32_t* agent_type, const float* W1,
+                                 const float* b1, const float* W_ih, const float* b_ih, const float* W_hh,
+                                 const float* b_hh, const float* W2, const float* b2, uint64_t version) {
+  if (!a) return fail(MARL_EINVAL, "actor is NULL");
+  if (!agent_type || !W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a pointer is NULL");
+  const marl_actor_config_t& c = a->cfg;
+  const int cap = c.n_agent_types > 1 ? c.n_agent_types : 1;
+  if (n_types < 1 || n_types > cap)
+    return fail(MARL_EINVAL, "n_types=%d, but the actor was created for at most %d (n_agent_types)", n_types, cap);
+  uint64_t bits = 0;
+  for (int i = 0; i < c.n_agents; ++i) {
+    if (agent_type[i] < 0 || agent_type[i] >= n_types)
+      return fail(MARL_EINVAL, "agent_type[%d]=%d is outside [0, %d)", i, agent_type[i], n_types);
+    bits |= (uint64_t)agent_type[i] << (2 * i);
+  }
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  if (a->pending) {
+    CU_TRY(cudaStreamSynchronize(a->copy_stream));
+    a->pending = false;
+  }
+  const int n = c.n_agents, D = c.obs_dim, A = c.n_actions, H = c.hidden, I = D + n + A;
+  const size_t tcb = tc_wpack_bytes(n, D, A, H);
+  a->host_pack.assign((size_t)n_types * a->wo.total + a->wo.total + tcb, 0);
+  std::vector<uint8_t> one(a->wo.total + tcb);
+  for (int k = 0; k < n_types; ++k) {  // the CUDA-core image of every type, one after the other
+    pack_weights_host(a, W1 + (size_t)k * H * I, b1 + (size_t)k * H, W_ih + (size_t)k * 3 * H * H, b_ih + (size_t)k * 3 * H,
+                      W_hh + (size_t)k * 3 * H * H, b_hh + (size_t)k * 3 * H, W2 + (size_t)k * A * H, b2 + (size_t)k * A,
+                      one.data());
+    memcpy(a->host_pack.data() + (size_t)k * a->wo.total, one.data(), a->wo.total);
+  }
+  CU_TRY(cudaMemcpyAsync(a->state + a->so.wff[a->wslot], a->host_pack.data(), (size_t)n_types * a->wo.total,
+                         cudaMemcpyHostToDevice, a->stream));
+  CU_TRY(cudaStreamSynchronize(a->stream));
+  a->weights_version = version;
+  a->have_weights = true;
+  a->n_types = n_types;
+  a->agent_type_bits = bits;
+  a->use_tc = a->use_tcp = false;  // per-type networks run on the CUDA-core kernel
+  if (n_types == 1) {              // a single type is the shared network: its tensor-core image as well
+    const int rc = upload_weights(a, one.data(), a->wslot, a->stream);
+    if (rc) return rc;
+    CU_TRY(cudaStreamSynchronize(a->stream));
+    a->use_tc = a->tc_allowed;
+    a->use_tcp = a->tcp_allowed;
+  }
   return MARL_OK;
 }
 
@@ -439,6 +502,7 @@ int marl_actor_publish_weights(marl_actor_t* a, const float* W1, const float* b1
   if (!a) return fail(MARL_EINVAL, "actor is NULL");
   if (!W1 || !b1 || !W_ih || !b_ih || !W_hh || !b_hh || !W2 || !b2) return fail(MARL_EINVAL, "a weight pointer is NULL");
   if (!a->have_weights) return fail(MARL_EINVAL, "marl_actor_set_weights has not been called");
+  if (a->n_types > 1) return fail(MARL_EINVAL, "per-type networks are loaded: publish is for the shared network only");
   if (effective_step < a->step) return fail(MARL_EINVAL, "effective_step %llu is already enqueued (next step is %llu)",
                                             (unsigned long long)effective_step, (unsigned long long)a->step);
   if (!a->copy_stream) {
@@ -499,6 +563,9 @@ static void fill_params(marl_actor* a, ActorParams& p) {
   p.env_ids = nullptr;
   p.M = c.n_envs;
   p.lagged = 0;
+  p.n_types = a->n_types;
+  p.type_stride = (uint32_t)(a->wo.total / sizeof(float));
+  p.agent_type_bits = a->agent_type_bits;
   p.trace_actions = a->trace_actions;
   p.trace_q = a->trace_q;
   p.trace_first = a->trace_next;

@@ -47,7 +47,10 @@ def run_gpu_rollout(cfg, weights, kernel="auto", T=None, splits=None, want_q=Tru
     the traced actions / Q as device tensors."""
     T = cfg["T"] if T is None else T
     actor = binding.Actor(cfg, kernel=kernel, work_steps=work_steps)
-    actor.set_weights(weights)
+    if isinstance(weights, dict):
+        actor.set_weights(weights)
+    else:                                   # one network per unit type
+        actor.set_weights_typed(weights)
     acts, q = actor.set_trace(T, want_q=want_q)
     for part in (splits or [T]):
         actor.rollout(cfg["env"], part, cfg["eps_start"], cfg["eps_end"], cfg["anneal_steps"])
