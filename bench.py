@@ -477,7 +477,8 @@ def main():
     bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T_launch) * E * n * T_launch
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     flop_rate = flops_per_agent_step(cfg) * E * n * T_launch / (kernel_ms * 1e-3) / 1e12
-    kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel"}.get(actor.kernel_name, "actor_ffma_kernel")
+    kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel",
+             "tcgen05-streamed": "actor_tcw_kernel"}.get(actor.kernel_name, "actor_ffma_kernel")
     if cfg["precision"] == "fp32":
         # the fp32 path is bound by plain FFMA arithmetic: peak measured on this device by the library's FMA loop
         ffma_peak = binding.marl_measure_ffma_tflops()

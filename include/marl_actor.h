@@ -55,8 +55,10 @@ extern "C" {
                               * shape is supported, at every batch size; otherwise, and for fp32, FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
-#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, hidden 64, at least 4 agents, n_agents * n_actions
-                                        * a multiple of 4; create fails otherwise.  Inputs that are not 16-byte
+#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, at least 4 agents; hidden 64 with n_agents * n_actions
+                                        * a multiple of 4, or hidden 128 with at most 16 actions, obs_dim a multiple of
+                                        * 8 and n_agents * n_actions a multiple of 16 (weights streamed from L2, dense
+                                        * launches only); create fails otherwise.  Inputs that are not 16-byte
                                         * aligned (or, where an environment's observation or availability block is
                                         * not a 16-byte multiple, an environment count that is not a multiple of 4)
                                         * fall back, per call, to the one-tile kernel where the shape allows it,
@@ -353,7 +355,8 @@ int marl_selftest_bounded_wait(void* stream, uint32_t poll_limit, uint32_t* stat
  * at the clocks it actually sustains.  SYNCHRONISES the stream; takes a few tens of milliseconds. */
 int marl_measure_ffma_tflops(void* stream, double* tflops_out);
 
-/* Name of the step kernel in use: "ffma", "tcgen05" (one-tile tensor-core kernel) or "tcgen05-pipelined". */
+/* Name of the step kernel in use: "ffma", "tcgen05" (one-tile tensor-core kernel), "tcgen05-pipelined", or
+ * "tcgen05-streamed" (hidden size 128: the pipelined design with the weights streamed through shared memory). */
 const char* marl_actor_kernel_name(const marl_actor_t* a);
 
 /* Launches of library kernels enqueued by this actor since creation (all kernels, all entry points). */

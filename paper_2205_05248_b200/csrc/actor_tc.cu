@@ -40,7 +40,13 @@ bool tc_supported(int n, int D, int A, int H, int prec) {
   return tc_layout(n, D, A, rec_bytes_of(n, D, A)).total <= TC_SMEM_MAX;
 }
 
+// (the packed image of the hidden-128 kernel: actor_tcw.cu)
+size_t tcw_wpack_bytes(int n, int D, int A);
+void tcw_pack_weights(int n, int D, int A, const float* W1, const float* b1, const float* Wih, const float* bih,
+                      const float* Whh, const float* bhh, const float* W2, const float* b2, void* dst_host);
+
 size_t tc_wpack_bytes(int n, int D, int A, int H) {
+  if (H == 128) return tcw_wpack_bytes(n, D, A);
   if (H != TC_H || D < 1 || D > 256 || n < 1 || n > 32 || A < 1 || A > 32) return 0;  // (a layout question only)
   return tc_layout(n, D, A, rec_bytes_of(n, D, A)).wbytes;
 }
@@ -65,6 +71,10 @@ static size_t operand_offset(int N, int row, int k) { return (size_t)(k / 8) * N
 void tc_pack_weights(int n, int D, int A, int H, const float* W1, const float* b1, const float* Wih,
                      const float* bih, const float* Whh, const float* bhh, const float* W2, const float* b2,
                      void* dst_host) {
+  if (H == 128) {
+    tcw_pack_weights(n, D, A, W1, b1, Wih, bih, Whh, bhh, W2, b2, dst_host);
+    return;
+  }
   const TcLayout L = tc_layout(n, D, A, rec_bytes_of(n, D, A));
   const int I = D + n + A;
   uint8_t* o = static_cast<uint8_t*>(dst_host);

@@ -28,6 +28,8 @@ void tc_tiling(int E, int n, int sms, int* ept, int* num_tiles);
 int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream);
 bool tcp_supported(int n, int D, int A, int H, int prec);
 int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream);
+bool tcw_supported(int n, int D, int A, int H, int prec);
+int launch_actor_tcw(const ActorParams& p, int sms, cudaStream_t stream);
 int launch_ring_sample(const SampleParams& p, cudaStream_t stream);
 }  // namespace marl
 
@@ -301,7 +303,8 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   a->pending_version = a->pending_step = 0;
 
   const bool tc_ok = tc_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
-  const bool tcp_ok = tcp_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
+  const bool tcp_ok = tcp_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision) ||
+                      tcw_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
   if ((cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) || (cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED && !tcp_ok)) {
     delete a;
     return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
@@ -411,7 +414,8 @@ static void pack_weights_host(marl_actor* a, const float* W1, const float* b1, c
   memcpy(hp + a->wo.bih, b_ih, sizeof(float) * 3 * H);
   memcpy(hp + a->wo.bhh, b_hh, sizeof(float) * 3 * H);
   memcpy(hp + a->wo.b2, b2, sizeof(float) * A);
-  if (tcb && (tc_supported(n, D, A, H, a->cfg.precision) || tcp_supported(n, D, A, H, a->cfg.precision)))
+  if (tcb && (tc_supported(n, D, A, H, a->cfg.precision) || tcp_supported(n, D, A, H, a->cfg.precision) ||
+              tcw_supported(n, D, A, H, a->cfg.precision)))
     tc_pack_weights(n, D, A, H, W1, b1, W_ih, b_ih, W_hh, b_hh, W2, b2, hp + a->wo.total);
 }
 
@@ -624,7 +628,8 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   int rc = 0;
   if (a->use_tcp || a->use_tc) {
     tc_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
-    if (a->use_tcp) rc = launch_actor_tcp(p, a->sms, a->stream);   // 0: these pointers cannot be bulk-copied
+    if (a->use_tcp)  // 0: these pointers cannot be bulk-copied
+      rc = c.hidden == 128 ? launch_actor_tcw(p, a->sms, a->stream) : launch_actor_tcp(p, a->sms, a->stream);
     // (the one-tile kernel bulk-copies the observations too; it copes with unaligned availability bytes itself)
     if (rc == 0 && a->use_tc && reinterpret_cast<uintptr_t>(obs) % 16 == 0) rc = launch_actor_tc(p, a->sms, a->stream);
   }
@@ -708,7 +713,7 @@ static int step_list(marl_actor* a, const int32_t* env_ids, int32_t M, const flo
   int rc = 0;
   if (a->use_tcp) {  // 0: these pointers or this list length cannot be bulk-copied
     tc_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
-    rc = launch_actor_tcp(p, a->sms, a->stream);
+    rc = c.hidden == 128 ? 0 : launch_actor_tcp(p, a->sms, a->stream);  // (the hidden-128 kernel takes dense launches only)
   }
   if (rc == 0) {
     ffma_tiling(M, c.n_agents, a->sms, &p.ept, &p.num_tiles);
@@ -933,7 +938,8 @@ int marl_actor_reset(marl_actor_t* a) {
 
 const char* marl_actor_kernel_name(const marl_actor_t* a) { 
   if (!a) return "ffma";
-  return a->use_tcp ? "tcgen05-pipelined" : (a->use_tc ? "tcgen05" : "ffma");
+  if (a->use_tcp) return a->cfg.hidden == 128 ? "tcgen05-streamed" : "tcgen05-pipelined";
+  return a->use_tc ? "tcgen05" : "ffma";
 }
 
 uint64_t marl_actor_launch_count(const marl_actor_t* a) { return a ? a->launches : 0; }

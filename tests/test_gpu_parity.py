@@ -72,12 +72,15 @@ def test_configs_2_to_4_parity(k, n_ids):
 
 
 @pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "pipelined"), (64, "bf16", "tensor"), (64, "bf16", "ffma"),
-                                           (128, "bf16", "ffma"), (64, "fp32", "ffma"), (128, "fp32", "ffma")])
+                                           (128, "bf16", "auto"), (128, "bf16", "ffma"), (64, "fp32", "ffma"),
+                                           (128, "fp32", "ffma")])
 def test_config5_parity_small_E(H, prec, kernel):
     cfg = workloads.config(5, E=4096, H=H, precision=prec)
     cfg["T"] = 24
     w = workloads.make_weights(cfg)
     actor, acts, q = run_gpu_rollout(cfg, w, kernel=kernel)
+    if kernel == "auto":
+        assert actor.kernel_name == ("tcgen05-streamed" if H == 128 else "tcgen05-pipelined")
     res = referee(cfg, w, actor, acts, q)          # every environment
     print(f"cfg5 H={H} {prec} {kernel}: {res}")
     actor.destroy()
@@ -494,3 +497,44 @@ def test_guard_bytes_around_the_buffers_catch_a_stray_write():
             actor.check_guards()
         full[where] = keep
     actor.destroy()
+
+
+def test_streamed_hidden128_kernel_shapes_episode_ends_and_split_launches():
+    """The tensor-core kernel for hidden size 128 (weights streamed through shared memory): tile tails, partial staging
+    chunks, one tile, more tiles than blocks, agent counts that do not divide 128, observation widths that need padding
+    to the MMA's K step; an episode end in every step and never; launches of one step and split rollouts."""
+    for over in (dict(E=130, n=8, D=80, A=14, C=260), dict(E=1, n=4, A=4, D=8, C=2), dict(E=37, n=16, A=5, D=16, C=74),
+                 dict(E=9, n=32, A=2, D=40, C=9), dict(E=2500, n=8, A=6, D=72, C=2500), dict(E=333, n=12, A=4, D=88, C=333)):
+        cfg = workloads.small_config(H=128, L=7, T=20, precision="bf16", **over)
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w, kernel="pipelined", splits=[1, 6, 13])
+        assert actor.kernel_name == "tcgen05-streamed"
+        res = referee(cfg, w, actor, acts, q)
+        print(f"H=128 {over}: {res}")
+        actor.destroy()
+    for thr, L in ((1 << 24, 4), (0, 5)):
+        cfg = workloads.small_config(H=128, D=8, E=40, n=4, A=8, C=80, L=L, T=17, precision="bf16", env=dict(done_thresh24=thr))
+        w = workloads.make_weights(cfg)
+        actor, acts, q = run_gpu_rollout(cfg, w)
+        assert actor.kernel_name == "tcgen05-streamed"
+        referee(cfg, w, actor, acts, q)
+        _, counters = actor.status()
+        assert counters["episodes"] == (40 * 17 if thr else 40 * (17 // 5))
+        actor.destroy()
+    # step calls (one-step launches) reproduce the rollout; a list step falls back to the CUDA-core kernel and is clean
+    cfg = workloads.small_config(H=128, D=24, E=50, n=4, A=12, C=100, L=8, T=12, precision="bf16")
+    w = workloads.make_weights(cfg)
+    ref, acts, q = run_gpu_rollout(cfg, w)
+    obs, avail, rew, done = ref.env_generate(cfg["env"], 0, cfg["T"])
+    dev = binding.Actor(cfg)
+    dev.set_weights(w)
+    for t in range(cfg["T"]):
+        assert torch.equal(dev.step(obs[t], avail[t], rew[t], done[t], cfg["eps_start"]), acts[t])
+    torch.cuda.synchronize()
+    assert torch.equal(dev.ring_mem, ref.ring_mem)
+    ids = np.arange(0, 48, 2, dtype=np.int32)
+    tid = torch.as_tensor(ids, device="cuda", dtype=torch.long)
+    dev.step_subset(ids, *(x[0].index_select(0, tid).contiguous() for x in (obs, avail, rew, done)), 0.1)
+    assert dev.status()[0] == 0
+    ref.destroy()
+    dev.destroy()
