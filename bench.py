@@ -79,13 +79,15 @@ def flops_per_agent_step(cfg: dict) -> float:
     return 2.0 * H * (D + 6 * H + A) + 25.0 * H
 
 
-def measured_traffic(kernel_name: str, agent_steps_per_launch: float):
-    """DRAM bytes per launch from the committed ncu record of this kernel, or None if there is no record or the
-    kernel sources have changed since the counters were taken."""
+def traffic_record(kernel_name: str, agent_steps_per_launch: float, algorithmic_bytes: float) -> dict:
+    """DRAM bytes per launch from the committed ncu record of this kernel: {"traffic": bytes or None, ...}.  None if
+    there is no record or the kernel sources have changed since the counters were taken.  The record comes from a
+    small case and is scaled by the agent-steps of a launch; where the scaled figure falls below the algorithmic
+    bytes (the small case ends with part of its last writes still in L2), it is a lower bound and says so."""
     import hashlib
     path = os.path.join(ROOT, "profiles", f"{kernel_name}_traffic.txt")
     if not os.path.exists(path):
-        return None
+        return {"traffic": None}
     rec = {}
     for line in open(path):
         if line.startswith("#") or ":" not in line:
@@ -97,10 +99,14 @@ def measured_traffic(kernel_name: str, agent_steps_per_launch: float):
         for f in rec["source_files"].split():
             h.update(open(os.path.join(ROOT, f), "rb").read())
         if h.hexdigest() != rec["source_sha256"]:
-            return None
-        return float(rec["dram_bytes_per_agent_step"]) * agent_steps_per_launch
+            return {"traffic": None}
+        scaled = float(rec["dram_bytes_per_agent_step"]) * agent_steps_per_launch
     except (KeyError, OSError, ValueError):
-        return None
+        return {"traffic": None}
+    note = (f"ncu capture of {rec.get('capture_agent_steps', '?')} agent-steps scaled to one launch"
+            + ("; below the algorithmic bytes: a lower bound (the small case ends with writes still in L2)"
+               if scaled < algorithmic_bytes else ""))
+    return {"traffic": scaled, "traffic_note": note}
 
 
 def load_peaks():
@@ -487,11 +493,22 @@ def main():
                     "kernel": kname, "kernel_ms": kernel_ms, "flops_per_agent_step": flops_per_agent_step(cfg),
                     "hbm_gbs_achieved": achieved}
     else:
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": measured_traffic(kname, E * n * T_launch),
-                    "peak_source": peak_kind, "kernel": kname,
-                    "kernel_ms": kernel_ms, "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T_launch),
-                    "tflops_effective": flop_rate}
+        # The step's roofline is the slower of its bytes at the measured HBM bandwidth and its FLOPs at the measured
+        # bf16 tensor throughput (the sustained figure: the timed region is a loop of seconds).
+        tf_peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
+        t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
+        t_tensor = flops_per_agent_step(cfg) * E * n * T_launch / (tf_peak * 1e12)
+        common = {"peak_source": peak_kind, "kernel": kname, "kernel_ms": kernel_ms,
+                  "algorithmic_bytes_per_agent_step": algorithmic_bytes_per_agent_step(cfg, T_launch),
+                  "flops_per_agent_step": flops_per_agent_step(cfg), "hbm_gbs_achieved": achieved,
+                  "tflops_effective": flop_rate, "hbm_frac": achieved / peaks["hbm_gbs"], "tensor_frac": flop_rate / tf_peak}
+        if t_tensor > t_hbm:
+            roofline = {"bound": "tensor", "achieved": flop_rate, "peak": tf_peak, "unit": "TFLOP/s",
+                        "frac": flop_rate / tf_peak, "traffic": None, **common}
+        else:
+            roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": achieved / peaks["hbm_gbs"], **traffic_record(kname, E * n * T_launch, bytes_per_launch),
+                        **common}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "ms_per_step_median": ms_median,
