@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--E", type=int, default=None)
     ap.add_argument("--H", type=int, default=None)
     ap.add_argument("--precision", default=None, choices=[None, "fp32", "bf16"])
-    ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor", "pipelined"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "ffma", "tensor", "pipelined", "dual"])
     ap.add_argument("--refresh", action="store_true",
                     help="publish a new network during every step, effective at the middle of the next rollout "
                          "(the learner's model update running beside the workers)")
@@ -483,7 +483,7 @@ def main():
     bytes_per_launch = algorithmic_bytes_per_agent_step(cfg, T_launch) * E * n * T_launch
     achieved = bytes_per_launch / (kernel_ms * 1e-3) / 1e9
     flop_rate = flops_per_agent_step(cfg) * E * n * T_launch / (kernel_ms * 1e-3) / 1e12
-    kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel",
+    kname = {"tcgen05-pipelined": "actor_tcp_kernel", "tcgen05": "actor_tc_kernel", "tcgen05-dual": "actor_tc2_kernel",
              "tcgen05-streamed": "actor_tcw_kernel"}.get(actor.kernel_name, "actor_ffma_kernel")
     if cfg["precision"] == "fp32":
         # the fp32 path is bound by plain FFMA arithmetic: peak measured on this device by the library's FMA loop

@@ -51,8 +51,8 @@ extern "C" {
 #define MARL_PRECISION_FP32 0 /* fp32 weights, fp32 FFMA arithmetic */
 #define MARL_PRECISION_BF16 1 /* weight matrices and matmul operands rounded to bf16 (RNE), fp32 accumulate */
 
-#define MARL_KERNEL_AUTO 0   /* bf16: a tensor-core kernel (the pipelined one where the shape allows it) wherever the
-                              * shape is supported, at every batch size; otherwise, and for fp32, FFMA */
+#define MARL_KERNEL_AUTO 0   /* bf16: a tensor-core kernel (the pipelined one, else the one-tile one, as the shape allows)
+                              * wherever the shape is supported, at every batch size; otherwise, and for fp32, FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
 #define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, at least 4 agents; hidden 64 with n_agents * n_actions
@@ -65,6 +65,13 @@ extern "C" {
                                         * else to the FFMA kernel */
 
 #define MARL_MAX_AGENT_TYPES 4
+
+#define MARL_KERNEL_TENSOR_DUAL 4 /* the pipelined design with two tiles of environments resident per SM (never chosen
+                                  * automatically: it measures slower than the pipelined kernel): bf16, hidden 64,
+                                  * 5 to 32 agents, at most 16 actions, obs_dim a multiple of 8, n_agents * n_actions
+                                  * a multiple of 16; create fails otherwise.  Launches it does not take (fewer than 8
+                                  * steps, no more tiles than SMs, list steps, unaligned inputs) run on the pipelined
+                                  * kernel; results are identical bit for bit */
 
 #define MARL_STATUS_NO_AVAIL 1u  /* some row had no available action (action 0 was taken) */
 #define MARL_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; results of that launch are invalid */
@@ -355,7 +362,8 @@ int marl_selftest_bounded_wait(void* stream, uint32_t poll_limit, uint32_t* stat
  * at the clocks it actually sustains.  SYNCHRONISES the stream; takes a few tens of milliseconds. */
 int marl_measure_ffma_tflops(void* stream, double* tflops_out);
 
-/* Name of the step kernel in use: "ffma", "tcgen05" (one-tile tensor-core kernel), "tcgen05-pipelined", or
+/* Name of the step kernel in use: "ffma", "tcgen05" (one-tile tensor-core kernel), "tcgen05-pipelined",
+ * "tcgen05-dual" (two resident tiles; its other launches run on the pipelined kernel), or
  * "tcgen05-streamed" (hidden size 128: the pipelined design with the weights streamed through shared memory). */
 const char* marl_actor_kernel_name(const marl_actor_t* a);
 

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmarl_actor.so")
 
 PRECISION = {"fp32": 0, "bf16": 1}
-KERNEL = {"auto": 0, "ffma": 1, "tensor": 2, "pipelined": 3}
+KERNEL = {"auto": 0, "ffma": 1, "tensor": 2, "pipelined": 3, "dual": 4}
 STATUS_NO_AVAIL, STATUS_TIMEOUT, STATUS_BAD_INDEX = 1, 2, 4
 
 # Debug aid: with GUARD_BYTES > 0 (a multiple of 256; the test-suite sets it) every buffer an Actor hands to the

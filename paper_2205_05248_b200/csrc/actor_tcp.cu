@@ -39,20 +39,6 @@
 
 namespace marl {
 
-// Phase timeline for tuning (compiled in only with -DMARL_TP_STAMPS): block 0 records the SM clock at its
-// hand-offs, per step, for a host-side reader.
-#ifdef MARL_TP_STAMPS
-__device__ unsigned long long g_tp_stamp[256 * 32];
-#define TP_STAMP(cond, step, id)                                                              \
-  do {                                                                                        \
-    if ((cond) && blockIdx.x == 0 && (step) < 256u) g_tp_stamp[(step) * 32 + (id)] = clock64(); \
-  } while (0)
-#else
-#define TP_STAMP(cond, step, id) \
-  do {                           \
-  } while (0)
-#endif
-
 constexpr int TP_THREADS = 512;
 constexpr int TP_CONV = 128;          // converter threads
 constexpr int TP_G = 4;               // environments per staging chunk
@@ -316,18 +302,15 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           } else {
             mbar_wait(&B->stepd, par ^ 1u, abortf);
           }
-          TP_STAMP(lane == 0, (uint32_t)g, 15);
           tp_issue_hside<NQ>(L, sb, tmem, lane, qcol);
         }
         mbar_wait(&B->yready, par, abortf);
-        TP_STAMP(lane == 0, (uint32_t)g, 8);
         tc_fence_after_sync();
         if (lane == 0) {
           const uint64_t d_y = smem_desc(sb + L.off_y, TC_LBO_A, 128), d_Wih = smem_desc(sb + L.off_Wih, TP_LBO_G, 128);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) mma_bf16(tmem + TM_R, d_y + ks * TP_K_A, d_Wih + ks * TP_K_G, idesc_bf16_f32(128, 192), 1);
           mma_commit(&B->grud);
-          TP_STAMP(true, (uint32_t)g, 9);
         }
         __syncwarp();
         // fc1 of the next step (possibly the next tile's first): its accumulator is free since epilogue 1 of
@@ -338,12 +321,10 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const uint32_t ready = __shfl_sync(0xFFFFFFFFu, lane == 0 ? (uint32_t)mbar_test_wait(&B->xready, par ^ 1u) : 0u, 0);
           if (ready) {
             tp_issue_fc1(L, sb, tmem, lane, &B->fc1d);
-            TP_STAMP(lane == 0, (uint32_t)g, 10);
             pending = false;
           }
         }
         mbar_wait(&B->hready, par, abortf);
-        TP_STAMP(lane == 0, (uint32_t)g, 11);
         tc_fence_after_sync();
         if (lane == 0) {
           const uint64_t d_h = smem_desc(sb + L.off_hb, TC_LBO_A, 128), d_W2 = smem_desc(sb + L.off_W2, NQ * 16, 128);
@@ -352,13 +333,11 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             mma_bf16(tmem + qcol + (NQ == 16 ? ks * NQ : 0), d_h + ks * TP_K_A, d_W2 + ks * ((2 * NQ * 16) >> 4), idesc_bf16_f32(128, NQ),
                      (NQ == 16 && ks > 0) ? 0 : 1);
           mma_commit(&B->fc2d);
-          TP_STAMP(true, (uint32_t)g, 12);
         }
         __syncwarp();
         if (pending) {
           mbar_wait(&B->xready, par ^ 1u, abortf);
           tp_issue_fc1(L, sb, tmem, lane, &B->fc1d);
-          TP_STAMP(lane == 0, (uint32_t)g, 13);
         }
         // The next step's h-side products need only the new hidden state, which is in place unless an episode
         // of this tile ends with this step (its rows are cleared after fc2): issue them now, off the critical
@@ -370,7 +349,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           // (published by the load warp before this step's inputs were requested: ordered before the fc1 operand)
           if (closeany_s[g & (TP_DST_DEPTH - 1)] == 0) {
             tp_issue_hside<NQ>(L, sb, tmem, lane, TM_Q + (par ^ 1u) * tp_qstride(NQ));
-            TP_STAMP(lane == 0, (uint32_t)g, 14);
             hside_issued = true;
           }
         }
@@ -522,14 +500,12 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&B->flags);  // first: epilogue 3 of this step waits for it
-          TP_STAMP(lane == 0, it, 21);
           if (s > 0) copy_tails(b ^ 1u);           // then the previous step's tails, off the critical path
           if (mine && s + 1 < T) {
             reward_next = p.reward[(size_t)(s + 1) * p.env_step_stride + x];
             done_next = p.done[(size_t)(s + 1) * p.env_step_stride + x];
           }
           mbar_wait(&B->stepd, sd & 1, abortf);  // action and Q of step s are in the tail
-          TP_STAMP(lane == 0, it, 20);
           ++sd;
           tdst_s[lane] = dst;
           if (close) {
@@ -613,7 +589,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         uint2* sel = sel_s + (it & 3) * TC_ROWS;
         // the operand buffer is free once fc1 of the previous step has finished reading it
         if (it > 0) mbar_wait(&B->fc1d, (it - 1) & 1, abortf);
-        TP_STAMP(ci == 0, it, 16);
         for (int c = cw; c < nck; c += TP_CONV / 32) {
           const int ge = min(TP_G, ne - c * TP_G);
           const int Rc = ge * n;         // rows of this chunk
@@ -707,7 +682,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         qbase += (uint32_t)nck;
         fence_proxy_async_smem();
         warp_arrive(&B->xready, lane);
-        TP_STAMP(ci == 0, it, 17);
         asm volatile("bar.sync 2, 128;" ::: "memory");  // the masks were written by the chunks' warps
         if (ci < ne * n) {
           const int rel = ci / n, rai = ci - rel * n;
@@ -718,7 +692,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           sel[ci].y = (uint32_t)pick;
         }
         warp_arrive(&B->selready[it & 3], lane);
-        TP_STAMP(ci == 0, it, 18);
         ++it;
       }
     }
@@ -752,7 +725,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 
       // ---- tile prologue: hidden state and last actions from global memory ----
       {
-        TP_STAMP(tid == 0, it, 22);
         bool carry = live;  // the row continues an episode
         if (LAG && live) {  // ... unless the late outcome has just ended it
           const int ps = p.pos[e];
@@ -812,7 +784,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
                                      pack_bf16x2(h[8 * cc + 4], h[8 * cc + 5]), pack_bf16x2(h[8 * cc + 6], h[8 * cc + 7]));
           *reinterpret_cast<uint4*>(hb + (uint32_t)(half * 4 + cc) * TC_LBO_A + (uint32_t)row * 16u) = o;
         }
-        TP_STAMP(tid == 0, it, 23);
         if (half == 0) {
           la = la_mem;
           if (la >= A) la = -1;
@@ -820,9 +791,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
-        TP_STAMP(tid == 0, it, 24);
         asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s is read by both threads of a row
-        TP_STAMP(tid == 0, it, 25);
         warp_arrive(&B->tiled, lane);
         // The next tile's hidden state is a first touch of its lines (and often of its page): ask for it now, one
         // line per thread, so that the next prologue finds it in L2.
@@ -844,7 +813,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         // ---- epilogue 1: y = relu(fc1 + W1[:, last action]) -> bf16 operand.  Bias and agent-id column are
         //      inside the GEMM; fc1 itself finished during the previous step. ----
         mbar_wait(&B->fc1d, par, abortf);
-        TP_STAMP(tid == 0, it, 0);
         tc_fence_after_sync();
         {
           // an episode that just ended has no last action
@@ -879,12 +847,10 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->yready, lane);
-        TP_STAMP(tid == 0, it, 1);
 
         // ---- epilogue 2: gate math, new hidden state (fp32 registers) and its bf16 operand.
         //      The r and z accumulators hold half the pre-activation: sigmoid(v) = 0.5 * tanh(v / 2) + 0.5 ----
         mbar_wait(&B->grud, par, abortf);
-        TP_STAMP(tid == 0, it, 2);
         tc_fence_after_sync();
         {
           // Eight columns at a time; the accumulators of the next eight are requested before the gate math of the
@@ -920,13 +886,10 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->hready, lane);
-        TP_STAMP(tid == 0, it, 3);
 
         // ---- epilogue 3: the row owners choose and complete the record's tail ----
         mbar_wait(&B->flags, par, abortf);  // close flags of this step written, tail buffer free
-        TP_STAMP(tid == 0, it, 19);
         mbar_wait(&B->fc2d, par, abortf);   // (both halves: the hidden operand may be cleared below)
-        TP_STAMP(tid == 0, it, 4);
         tc_fence_after_sync();
         if (half == 0) {
           uint32_t qv[NQ];
@@ -947,7 +910,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           tc_fence_before_sync();
           if (is_row) {
             mbar_wait(&B->selready[it & 3], (it >> 2) & 1, abortf);
-            TP_STAMP(tid == 0, it, 5);
             const uint2 sp = sel_s[(it & 3) * TC_ROWS + row];
             const uint32_t mask = sp.x;
             const int pick = (int)sp.y;
@@ -1001,7 +963,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           }
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        TP_STAMP(tid == 0, it, 6);
         // ---- a closed episode restarts from a zero hidden state and no last action ----
         if (live && close_s[b * 32 + el]) {
 #pragma unroll
@@ -1014,7 +975,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
         fence_proxy_async_smem();
         tc_fence_before_sync();
         warp_arrive(&B->stepd, lane);
-        TP_STAMP(tid == 0, it, 7);
         ++it;
       }
 
@@ -1045,7 +1005,6 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 #pragma unroll
         for (int q = 0; q < 8; ++q) dsth[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
       }
-      TP_STAMP(tid == 0, it, 26);
       asm volatile("bar.sync 1, 256;" ::: "memory");  // la_s is rewritten by the next tile's prologue
     }
     if (c_steps) atomicAdd(p.counters + CNT_AGENT_STEPS, c_steps);
@@ -1097,9 +1056,3 @@ int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
 }
 
 }  // namespace marl
-
-#ifdef MARL_TP_STAMPS
-extern "C" int marl_tp_stamps(unsigned long long* out_host) {
-  return (int)cudaMemcpyFromSymbol(out_host, marl::g_tp_stamp, sizeof(unsigned long long) * 256 * 32);
-}
-#endif

@@ -8,13 +8,13 @@
 // the ring records, a tail warp for headers, counters and the [action | Q | reward, done] part.
 //
 // What hidden size 128 changes:
-//   * The bf16 network is 228 KB and does not fit one SM's shared memory.  Only the bias tiles and the last-action
-//     table (23 KB) are resident; the four matrices are packed in global memory as a sequence of slices (at most
-//     12 KB each: one to three K = 16 steps of one matrix) in the order the tensor core consumes them, and a loader
-//     warp streams them from L2 through a ring of shared-memory slots, one bulk load per slice, as far ahead as the
-//     ring allows.  The thread that issues the MMAs waits for a slice, issues the MMAs that read it and hands the
-//     slot back with a tcgen05.commit.  Order per step: h-side r|z products, h-side candidate product, y-side
-//     products, fc2, fc1 of the next step.
+//   * The bf16 network is 228 KB and does not fit one SM's shared memory.  The bias tiles, the candidate rows of W_hh,
+//     W2 and the last-action table (60 KB) are resident; W1, W_ih and the reset/update rows of W_hh (185 KB) are packed
+//     in global memory as a sequence of slices (at most 12 KB each: one to three K = 16 steps of one matrix) in the
+//     order the tensor core consumes them, and a loader warp streams them from L2 through a ring of shared-memory
+//     slots, one bulk load per slice, as far ahead as the ring allows.  The thread that issues the MMAs waits for a
+//     slice, issues the MMAs that read it and hands the slot back with a tcgen05.commit.  Order per step: h-side r|z
+//     products, h-side candidate product, y-side products, fc2, fc1 of the next step.
 //   * Four 128-column accumulators (reset, update, candidate-input, candidate-hidden) fill tensor memory, so the
 //     fc1 accumulator lives in the candidate-input columns (issued once the gate math has read them) and Q in the
 //     candidate-hidden columns (read before the next step's candidate-hidden product is issued).
@@ -55,12 +55,12 @@ constexpr uint32_t TW_R = 0, TW_Z = 128, TW_IN = 256, TW_HN = 384, TW_COLS = 512
 
 struct TwLayout {
   int32_t Dk, nchunk, ept, ohK, ohc, NS, NW, n_slices;
-  int32_t ks_obs, ks_oh, nC, nE, pad0, pad1;          // K-steps of fc1; slices of the fc1 and candidate-hidden groups
+  int32_t ks_obs, ks_oh, nC, pad0, pad1, pad2;         // K-steps of fc1; slices of the fc1 group
   uint32_t slice_off[TW_MAX_SLICES];                  // byte offset of a slice inside the streamed image
   uint32_t slice_bytes[TW_MAX_SLICES];
   // packed weights in global memory: [resident image | streamed image]; the resident part has the same offsets in
   // shared memory
-  uint32_t off_Brz, off_Bin, off_Bhn, off_tab_la, rbytes, stream_off, wbytes;
+  uint32_t off_Brz, off_Bin, off_Bhn, off_Whn, off_W2, off_tab_la, rbytes, stream_off, wbytes;
   uint32_t prefix_bytes, tail_bytes, chunk_bytes, obs_bytes, av_bytes;
   uint32_t off_x, off_y, off_hb, off_oh, off_tail, off_sel, off_la, off_close, off_closeany, off_rowenv, off_dstp, off_tdst,
       off_bar, off_wring, off_stage, total;
@@ -74,13 +74,16 @@ struct TwBars {
   uint32_t tmem_base, abort;
 };
 
-// Streamed groups, in the order of use within a step (fc1 belongs to the NEXT step):
+// Resident: the bias tiles, the candidate rows of W_hh (32 KB), W2 (4.5 KB) and the last-action table.  Streamed
+// groups, in the order of use within a step (fc1 belongs to the NEXT step):
 //   D  W_hh rows r|z   (256 rows, K = 128): one K-step (8192 B) per slice
-//   E  W_hh rows n     (128 rows):          three K-steps (12288 B) per slice
 //   A  W_ih all rows   (384 rows):          one K-step (12288 B) per slice
-//   B  W2 + bias step  (16 rows, K = 144):  one slice (4608 B)
 //   C  W1              (128 rows, K = Dk + ohK): three K-steps (12288 B) per slice
-// The stream starts with C (fc1 of the first step), then D E A B C repeat.
+// The stream starts with C (fc1 of the first step), then D A C repeat: 185 KB per tile-step.  Every kilobyte of
+// shared memory is worth the same whether it keeps weights resident (less to stream) or deepens the ring (more
+// streamed while the gate math holds tensor memory): measured, the L2-to-SM stream runs at about 19 bytes per
+// clock and SM whatever the ring depth (2, 3 or 4 slots: 4.20, 3.98, 3.95 ms per rollout at 16384 environments),
+// so the ring is two slots and the rest holds weights.
 static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   TwLayout L;
   memset(&L, 0, sizeof(L));
@@ -96,6 +99,8 @@ static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   L.off_Brz = o; o += 2u * 256 * 16;
   L.off_Bin = o; o += 2u * 128 * 16;
   L.off_Bhn = o; o += 2u * 128 * 16;
+  L.off_Whn = o; o += 8u * 2 * 128 * 16;     // W_hh rows n (128 rows, K = 128): resident
+  L.off_W2 = o; o += 9u * 2 * TW_NQ * 16;    // W2 and its bias step (16 rows, K = 144): resident
   L.off_tab_la = o; o += up16((uint32_t)sizeof(float) * A * TW_TAB);
   L.rbytes = o;
   L.stream_off = o;
@@ -117,9 +122,7 @@ static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   };
   L.nC = add_group(L.ks_obs + L.ks_oh, 2u * 128 * 16, 3);  // C
   add_group(8, 2u * 256 * 16, 1);                           // D
-  L.nE = add_group(8, 2u * 128 * 16, 3);                    // E
   add_group(8, 2u * 384 * 16, 1);                           // A
-  add_group(1, 9u * 2 * TW_NQ * 16, 1);                     // B: nine K-steps in one slice
   L.n_slices = ns;
   L.wbytes = L.stream_off + so;
   // ---- shared memory ----
@@ -133,7 +136,7 @@ static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   L.off_y = o; o += 16 * TC_LBO_A;
   L.off_hb = o; o += 16 * TC_LBO_A;
   L.off_oh = o; o += (uint32_t)L.ohc * TC_LBO_A;
-  L.off_tail = o; o += 2u * (uint32_t)L.ept * L.tail_bytes;
+  L.off_tail = o; o += (uint32_t)L.ept * L.tail_bytes;
   L.off_sel = o; o += 4u * TC_ROWS * 8;
   L.off_la = o; o += TC_ROWS * 4;
   L.off_close = o; o += 2 * 32 * 4;
@@ -142,15 +145,19 @@ static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   L.off_dstp = o; o += TW_DST_DEPTH * 32 * 8;
   L.off_tdst = o; o += 32 * 8;
   L.off_bar = o; o += (uint32_t)((sizeof(TwBars) + 15) & ~15u);
-  // the staging ring holds one tile-step of chunks (so a slot's previous chunk always belongs to an earlier step),
-  // the weight ring takes what is left
+  // Two slots of weight ring; the staging ring takes what is left, up to one tile-step of chunks.  A staging ring
+  // shorter than a tile-step must be a multiple of the converter warps, so that the warp that waits for a slot is the
+  // one that converted the slot's previous chunk (a wait on "the other phase" reads as complete before that chunk
+  // has even arrived).
   const int nck_max = (L.ept + TW_G - 1) / TW_G;
-  L.NS = nck_max < 3 ? 3 : nck_max;
-  if (L.NS > TW_MAX_STAGES) L.NS = 0;
-  const uint32_t stage_bytes = (uint32_t)L.NS * L.chunk_bytes + 32;  // (+32: the mask words read a few bytes past a row)
-  const uint32_t used = o + stage_bytes;
-  int nw = used < TC_SMEM_MAX ? (int)((TC_SMEM_MAX - used) / TW_WSLOT) : 0;
-  if (nw > TW_MAX_WSLOTS) nw = TW_MAX_WSLOTS;
+  const int nw = 2;
+  const uint32_t fixed = o + (uint32_t)nw * TW_WSLOT + 32;  // (+32: the mask words read a few bytes past a row)
+  int nstage = fixed < TC_SMEM_MAX ? (int)((TC_SMEM_MAX - fixed) / L.chunk_bytes) : 0;
+  if (nstage > nck_max) nstage = nck_max < 3 ? 3 : nck_max;
+  if (nstage > TW_MAX_STAGES) nstage = TW_MAX_STAGES;
+  if (nstage < nck_max) nstage = nstage / TW_NCONV * TW_NCONV;
+  L.NS = nstage;
+  const uint32_t stage_bytes = (uint32_t)L.NS * L.chunk_bytes + 32;
   L.NW = nw;
   L.off_wring = o;
   L.off_stage = o + (uint32_t)nw * TW_WSLOT;
@@ -163,7 +170,7 @@ bool tcw_supported(int n, int D, int A, int H, int prec) {
   if (D < 1 || D > 256 || D % 8 != 0 || n < 4 || n > 32 || A < 1 || A > TW_NQ) return false;
   if ((n * A) % 16 != 0) return false;  // an environment's availability bytes are bulk-copied and stored as 16-byte pieces
   const TwLayout L = tw_layout(n, D, A, rec_bytes_of(n, D, A));
-  return L.ept >= TW_G && L.NS >= 3 && L.NW >= 3 && L.n_slices <= TW_MAX_SLICES && L.total <= TC_SMEM_MAX;
+  return L.ept >= TW_G && L.NS >= 3 && L.NW >= 2 && L.n_slices <= TW_MAX_SLICES && L.total <= TC_SMEM_MAX;
 }
 
 size_t tcw_wpack_bytes(int n, int D, int A) {
@@ -218,9 +225,8 @@ void tcw_pack_weights(int n, int D, int A, const float* W1, const float* b1, con
   uint32_t g = L.stream_off;
   const uint32_t gC = g; g += (uint32_t)(L.ks_obs + L.ks_oh) * 2u * 128 * 16;
   const uint32_t gD = g; g += 8u * 2 * 256 * 16;
-  const uint32_t gE = g; g += 8u * 2 * 128 * 16;
-  const uint32_t gA = g; g += 8u * 2 * 384 * 16;
-  const uint32_t gB = g;
+  const uint32_t gA = g;
+  const uint32_t gE = L.off_Whn, gB = L.off_W2;  // resident
   for (int j = 0; j < H; ++j) {
     for (int k = 0; k < D; ++k) put(gC, H, j, k, W1[(size_t)j * I + k]);
     put3(gC, H, j, L.Dk, b1[j]);
@@ -255,7 +261,7 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
   uint8_t* hb = smem + L.off_hb;
   uint8_t* oh = smem + L.off_oh;
   uint8_t* stage = smem + L.off_stage;
-  uint8_t* tails = smem + L.off_tail;                                  // [2][ept][tail_bytes]
+  uint8_t* tails = smem + L.off_tail;                                  // [ept][tail_bytes]
   uint2* sel_s = reinterpret_cast<uint2*>(smem + L.off_sel);          // [4][128]: availability mask, random pick or -1
   int32_t* la_s = reinterpret_cast<int32_t*>(smem + L.off_la);
   int32_t* close_s = reinterpret_cast<int32_t*>(smem + L.off_close);  // [2][32]
@@ -270,7 +276,6 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
   const int n = p.n, D = p.D, A = p.A, T = p.T;
   const uint32_t rec_bytes = p.rl.rec_bytes;
   const int NS = L.NS, NW = L.NW;
-  const uint32_t tail_set = (uint32_t)L.ept * L.tail_bytes;
   const uint32_t t_q = p.rl.off_q - p.rl.off_action, t_reward = p.rl.off_reward - p.rl.off_action,
                  t_done = p.rl.off_done - p.rl.off_action;
   const int my_tiles = blockIdx.x < p.num_tiles ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
@@ -380,19 +385,17 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
           slice_end();
         }
       };
-      // E: h-side product of the candidate, seeded with its bias
+      // h-side product of the candidate (resident weights), seeded with its bias
       auto issue_hside_n = [&]() {
         tc_fence_after_sync();
-        if (lane == 0)
+        if (lane == 0) {
           mma_bf16(tmem + TW_HN, smem_desc(sb + L.off_oh, TC_LBO_A, 128), smem_desc(sb + L.off_Bhn, 2048, 128), id128, 0);
-        for (int ks0 = 0; ks0 < 8; ks0 += 3) {
-          const uint32_t base = slice_begin();
-          if (lane == 0)
-            for (int j = 0; j < 3 && ks0 + j < 8; ++j)
-              mma_bf16(tmem + TW_HN, smem_desc(sb + L.off_hb, TC_LBO_A, 128) + (uint64_t)(ks0 + j) * K_A,
-                       smem_desc(base + (uint32_t)j * 4096u, 2048, 128), id128, 1);
-          slice_end();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            mma_bf16(tmem + TW_HN, smem_desc(sb + L.off_hb, TC_LBO_A, 128) + (uint64_t)ks * K_A,
+                     smem_desc(sb + L.off_Whn + (uint32_t)ks * 4096u, 2048, 128), id128, 1);
         }
+        __syncwarp();
       };
       if (total > 0) {
         mbar_wait(&B->xready, 0, abortf);
@@ -428,23 +431,21 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
         }
         if (lane == 0) mma_commit(&B->grud);
         __syncwarp();
-        // B: fc2 into four 16-column parts (dependent MMAs on one accumulator run one after the other): part ks % 4
-        // takes K-steps ks and ks + 4, part 0 starts from the bias step
+        // fc2 (resident weights) into four 16-column parts (dependent MMAs on one accumulator run one after the other):
+        // part ks % 4 takes K-steps ks and ks + 4, part 0 starts from the bias step
         mbar_wait(&B->hready, par, abortf);
         tc_fence_after_sync();
-        {
-          const uint32_t base = slice_begin();
-          if (lane == 0) {
-            const uint64_t dh = smem_desc(sb + L.off_hb, TC_LBO_A, 128);
-            mma_bf16(tmem + TW_HN, smem_desc(sb + L.off_oh, TC_LBO_A, 128), smem_desc(base + 8u * 512u, 256, 128), idq, 0);
+        if (lane == 0) {
+          const uint32_t base = sb + L.off_W2;
+          const uint64_t dh = smem_desc(sb + L.off_hb, TC_LBO_A, 128);
+          mma_bf16(tmem + TW_HN, smem_desc(sb + L.off_oh, TC_LBO_A, 128), smem_desc(base + 8u * 512u, 256, 128), idq, 0);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              mma_bf16(tmem + TW_HN + (uint32_t)(ks & 3) * 16u, dh + (uint64_t)ks * K_A, smem_desc(base + (uint32_t)ks * 512u, 256, 128), idq,
-                       (ks == 0 || ks >= 4) ? 1 : 0);
-            mma_commit(&B->fc2d);
-          }
-          slice_end();
+          for (int ks = 0; ks < 8; ++ks)
+            mma_bf16(tmem + TW_HN + (uint32_t)(ks & 3) * 16u, dh + (uint64_t)ks * K_A, smem_desc(base + (uint32_t)ks * 512u, 256, 128), idq,
+                     (ks == 0 || ks >= 4) ? 1 : 0);
+          mma_commit(&B->fc2d);
         }
+        __syncwarp();
         // C: fc1 of the next step (possibly the next tile's first): the gate math of this step has read the
         // candidate-input columns
         if (g + 1 < total) {
@@ -546,14 +547,17 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
           reward_next = p.reward[e];
           done_next = p.done[e];
         }
-        auto copy_tails = [&](uint32_t bb) {
+        // Copies the tails of the finished step (record addresses in tdst_s) to the ring: 16 bytes per lane, the
+        // pieces of all environments in one flat loop.  One tail buffer: the copy follows the step directly, and the
+        // next step's epilogue 3 is opened (flags) only after it.
+        auto copy_tails = [&]() {
           __syncwarp();
           const uint32_t pieces = L.tail_bytes / 16u, total = (uint32_t)ne * pieces;
           const uint32_t inv = 0xFFFFFFFFu / pieces + 1u;  // idx / pieces == umulhi(idx, inv) for idx < 2^16
           for (uint32_t idx = lane; idx < total; idx += 32) {
             const uint32_t env = __umulhi(idx, inv), pc = idx - env * pieces;
             const unsigned long long d = tdst_s[env];
-            if (d) reinterpret_cast<uint4*>(d)[pc] = reinterpret_cast<const uint4*>(tails + bb * tail_set + env * L.tail_bytes)[pc];
+            if (d) reinterpret_cast<uint4*>(d)[pc] = reinterpret_cast<const uint4*>(tails + env * L.tail_bytes)[pc];
           }
           __syncwarp();
         };
@@ -562,7 +566,7 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
           const float reward = reward_next;
           const int done = done_next ? 1 : 0;
           const int close = (ok && (done || pos + 1 == p.L)) ? 1 : 0;
-          uint8_t* tl = tails + b * tail_set + (uint32_t)lane * L.tail_bytes;
+          uint8_t* tl = tails + (uint32_t)lane * L.tail_bytes;
           unsigned long long dst = 0;
           close_s[b * 32 + lane] = close;
           if (mine && ok) {
@@ -576,8 +580,7 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
             tl[t_done] = (uint8_t)done;
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive(&B->flags);  // first: epilogue 3 of this step waits for it
-          if (s > 0) copy_tails(b ^ 1u);           // then the previous step's tails, off the critical path
+          if (lane == 0) mbar_arrive(&B->flags);  // epilogue 3 of this step may write the tails
           if (mine && s + 1 < T) {
             reward_next = p.reward[(size_t)(s + 1) * p.env_step_stride + e];
             done_next = p.done[(size_t)(s + 1) * p.env_step_stride + e];
@@ -585,6 +588,7 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
           mbar_wait(&B->stepd, sd & 1, abortf);  // action and Q of step s are in the tail
           ++sd;
           tdst_s[lane] = dst;
+          copy_tails();
           if (close) {
             p.slot_len[slot] = pos + 1;
             p.slot_complete[slot] = 1;
@@ -598,7 +602,6 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
           }
           ++it;
         }
-        copy_tails((it - 1) & 1);  // the tile's last step
         if (mine && ok) {
           p.slot[e] = slot;
           p.pos[e] = pos;
@@ -791,7 +794,7 @@ __global__ void __launch_bounds__(TW_THREADS, 1)
 
       for (int s = 0; s < T; ++s) {
         const uint32_t b = it & 1, par = it & 1;
-        uint8_t* tl = tails + b * tail_set + (uint32_t)el * L.tail_bytes;  // this row's environment tail
+        uint8_t* tl = tails + (uint32_t)el * L.tail_bytes;  // this row's environment tail
 
         // ---- epilogue 1: y = relu(fc1 + W1[:, last action]) -> bf16 operand (bias and agent-id column are inside
         //      the GEMM; the accumulator sits in the candidate-input columns) ----

@@ -28,6 +28,8 @@ void tc_tiling(int E, int n, int sms, int* ept, int* num_tiles);
 int launch_actor_tc(const ActorParams& p, int sms, cudaStream_t stream);
 bool tcp_supported(int n, int D, int A, int H, int prec);
 int launch_actor_tcp(const ActorParams& p, int sms, cudaStream_t stream);
+bool tc2_supported(int n, int D, int A, int H, int prec);
+int launch_actor_tc2(const ActorParams& p, int sms, cudaStream_t stream);
 bool tcw_supported(int n, int D, int A, int H, int prec);
 int launch_actor_tcw(const ActorParams& p, int sms, cudaStream_t stream);
 int launch_ring_sample(const SampleParams& p, cudaStream_t stream);
@@ -160,7 +162,7 @@ static int check_config(const marl_actor_config_t* c) {
     return fail(MARL_EINVAL, "ring_episodes must be a positive multiple of n_envs");
   if (c->precision != MARL_PRECISION_FP32 && c->precision != MARL_PRECISION_BF16)
     return fail(MARL_EINVAL, "unknown precision");
-  if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR_PIPELINED) return fail(MARL_EINVAL, "unknown kernel");
+  if (c->kernel < MARL_KERNEL_AUTO || c->kernel > MARL_KERNEL_TENSOR_DUAL) return fail(MARL_EINVAL, "unknown kernel");
   if (c->n_agent_types < 0 || c->n_agent_types > MARL_MAX_AGENT_TYPES)
     return fail(MARL_EINVAL, "n_agent_types must be in [0, %d]", MARL_MAX_AGENT_TYPES);
   if ((double)c->n_envs * c->n_agents > 1.0e9) return fail(MARL_EINVAL, "n_envs * n_agents too large");
@@ -173,7 +175,8 @@ struct marl_actor {
   int device, sms;
   bool use_tc;   // a tensor-core kernel steps this actor
   bool use_tcp;  // ... the pipelined one (falls back to the one-tile kernel for inputs it cannot bulk-copy)
-  bool tc_allowed, tcp_allowed;  // the choice made at creation; per-type networks switch the tensor-core kernels off
+  bool use_tc2;  // ... with two tiles resident per SM where a launch allows it (else the pipelined kernel, same results)
+  bool tc_allowed, tcp_allowed, tc2_allowed;  // the choice made at creation; per-type networks switch the tensor-core kernels off
   int32_t n_types;               // > 1: per-type networks are loaded
   uint64_t agent_type_bits;
   uint8_t *ring, *state, *work;
@@ -305,7 +308,9 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   const bool tc_ok = tc_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
   const bool tcp_ok = tcp_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision) ||
                       tcw_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision);
-  if ((cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) || (cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED && !tcp_ok)) {
+  const bool tc2_ok = tc2_supported(cfg->n_agents, cfg->obs_dim, cfg->n_actions, cfg->hidden, cfg->precision) && tcp_ok;
+  if ((cfg->kernel == MARL_KERNEL_TENSOR && !tc_ok) || (cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED && !tcp_ok) ||
+      (cfg->kernel == MARL_KERNEL_TENSOR_DUAL && !tc2_ok)) {
     delete a;
     return fail(MARL_EINVAL, "the tensor-core kernel does not support this shape/precision");
   }
@@ -314,8 +319,13 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   // rows to 16384 (`bench.py --crossover`, table in the benchmark spec), one 128-row tcgen05 tile takes 3.4-4.6 us per
   // environment step against 25-29 us for the CUDA-core kernel's 64-row tiles, so there is no batch size at which
   // the CUDA cores win.
-  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED || (cfg->kernel == MARL_KERNEL_AUTO && tcp_ok);
+  // (the two-tile kernel is never the automatic choice: measured at workload 5 it is slower than the pipelined kernel -
+  // 8.4 ms against 6.15 ms per 64-step rollout - because with the epilogue threads busy all the time the converter
+  // warps no longer keep up)
+  a->use_tc2 = cfg->kernel == MARL_KERNEL_TENSOR_DUAL;
+  a->use_tcp = cfg->kernel == MARL_KERNEL_TENSOR_PIPELINED || a->use_tc2 || (cfg->kernel == MARL_KERNEL_AUTO && tcp_ok);
   a->use_tc = tc_ok && cfg->kernel != MARL_KERNEL_FFMA;
+  a->tc2_allowed = a->use_tc2;
   a->tcp_allowed = a->use_tcp;
   a->tc_allowed = a->use_tc;
   a->n_types = 1;
@@ -449,6 +459,7 @@ int marl_actor_set_weights(marl_actor_t* a, const float* W1, const float* b1, co
   a->agent_type_bits = 0;
   a->use_tc = a->tc_allowed;
   a->use_tcp = a->tcp_allowed;
+  a->use_tc2 = a->tc2_allowed;
   return MARL_OK;
 }
 
@@ -489,13 +500,14 @@ int marl_actor_set_weights_typed(marl_actor_t* a, int32_t n_types, const int32_t
   a->have_weights = true;
   a->n_types = n_types;
   a->agent_type_bits = bits;
-  a->use_tc = a->use_tcp = false;  // per-type networks run on the CUDA-core kernel
+  a->use_tc = a->use_tcp = a->use_tc2 = false;  // per-type networks run on the CUDA-core kernel
   if (n_types == 1) {              // a single type is the shared network: its tensor-core image as well
     const int rc = upload_weights(a, one.data(), a->wslot, a->stream);
     if (rc) return rc;
     CU_TRY(cudaStreamSynchronize(a->stream));
     a->use_tc = a->tc_allowed;
     a->use_tcp = a->tcp_allowed;
+    a->use_tc2 = a->tc2_allowed;
   }
   return MARL_OK;
 }
@@ -628,7 +640,8 @@ static int enqueue_steps(marl_actor* a, const float* obs, const uint8_t* avail, 
   int rc = 0;
   if (a->use_tcp || a->use_tc) {
     tc_tiling(c.n_envs, c.n_agents, a->sms, &p.ept, &p.num_tiles);
-    if (a->use_tcp)  // 0: these pointers cannot be bulk-copied
+    if (a->use_tc2) rc = launch_actor_tc2(p, a->sms, a->stream);  // 0: not a launch for two resident tiles
+    if (rc == 0 && a->use_tcp)  // 0: these pointers cannot be bulk-copied
       rc = c.hidden == 128 ? launch_actor_tcw(p, a->sms, a->stream) : launch_actor_tcp(p, a->sms, a->stream);
     // (the one-tile kernel bulk-copies the observations too; it copes with unaligned availability bytes itself)
     if (rc == 0 && a->use_tc && reinterpret_cast<uintptr_t>(obs) % 16 == 0) rc = launch_actor_tc(p, a->sms, a->stream);
@@ -938,6 +951,7 @@ int marl_actor_reset(marl_actor_t* a) {
 
 const char* marl_actor_kernel_name(const marl_actor_t* a) { 
   if (!a) return "ffma";
+  if (a->use_tc2) return "tcgen05-dual";
   if (a->use_tcp) return a->cfg.hidden == 128 ? "tcgen05-streamed" : "tcgen05-pipelined";
   return a->use_tc ? "tcgen05" : "ffma";
 }

@@ -71,7 +71,7 @@ def test_configs_2_to_4_parity(k, n_ids):
     actor.destroy()
 
 
-@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "pipelined"), (64, "bf16", "tensor"), (64, "bf16", "ffma"),
+@pytest.mark.parametrize("H,prec,kernel", [(64, "bf16", "auto"), (64, "bf16", "dual"), (64, "bf16", "tensor"), (64, "bf16", "ffma"),
                                            (128, "bf16", "auto"), (128, "bf16", "ffma"), (64, "fp32", "ffma"),
                                            (128, "fp32", "ffma")])
 def test_config5_parity_small_E(H, prec, kernel):
@@ -93,7 +93,7 @@ def test_config5_full_size_bench_configuration():
     cfg = workloads.config(5)
     w = workloads.make_weights(cfg)
     actor = binding.Actor(cfg, kernel="auto", work_steps=1)
-    assert actor.kernel_name.startswith("tcgen05")
+    assert actor.kernel_name == "tcgen05-pipelined"
     actor.set_weights(w)
     acts, q = actor.set_trace(cfg["T"])
     staged = actor.env_generate(cfg["env"], 0, cfg["T"])
@@ -538,3 +538,32 @@ def test_streamed_hidden128_kernel_shapes_episode_ends_and_split_launches():
     assert dev.status()[0] == 0
     ref.destroy()
     dev.destroy()
+
+
+def test_two_resident_tiles_write_the_same_ring_as_the_pipelined_kernel():
+    """The kernel with two tiles resident per SM runs the arithmetic of the pipelined kernel: identical actions, Q,
+    records, headers and state, on batches of more tiles than SMs - an even and an odd number of tiles per block, a
+    ragged last tile, an episode end in every step, split launches (the short ones fall back to the pipelined kernel)."""
+    for over, env in ((dict(E=2400, n=8, D=80, A=14, C=2400), {}), (dict(E=4730, n=8, D=80, A=14, C=4730), {}),
+                      (dict(E=2500, n=16, D=24, A=5, C=5000), {}), (dict(E=5000, n=5, D=8, A=16, C=5000), dict(done_thresh24=1 << 24)),
+                      (dict(E=7001, n=6, D=40, A=8, C=7001), dict(done_thresh24=1 << 21))):
+        cfg = workloads.small_config(H=64, L=7, T=21, precision="bf16", env=env, **over)
+        w = workloads.make_weights(cfg)
+        a, acts_a, q_a = run_gpu_rollout(cfg, w, kernel="dual", splits=[9, 2, 10])
+        b, acts_b, q_b = run_gpu_rollout(cfg, w, kernel="pipelined", splits=[9, 2, 10])
+        assert a.kernel_name == "tcgen05-dual" and b.kernel_name == "tcgen05-pipelined"
+        assert torch.equal(acts_a, acts_b) and torch.equal(q_a, q_b), over        # bit for bit
+        assert torch.equal(a.ring_mem, b.ring_mem), over
+        sa, sb = a.get_state(), b.get_state()
+        for key in ("h", "last_action", "slot", "pos", "ep_count"):
+            assert torch.equal(sa[key], sb[key]), (over, key)
+        assert a.status() == b.status() and a.status()[0] == 0
+        a.destroy()
+        b.destroy()
+    # and against the oracle, every environment
+    cfg = workloads.small_config(H=64, L=9, T=24, precision="bf16", E=2600, n=8, D=80, A=14, C=5200)
+    w = workloads.make_weights(cfg)
+    actor, acts, q = run_gpu_rollout(cfg, w, kernel="dual")
+    res = referee(cfg, w, actor, acts, q)
+    print(f"dual: {res}")
+    actor.destroy()
