@@ -153,7 +153,8 @@ static TwLayout tw_layout(int n, int D, int A, int rec_bytes) {
   const int nw = 2;
   const uint32_t fixed = o + (uint32_t)nw * TW_WSLOT + 32;  // (+32: the mask words read a few bytes past a row)
   int nstage = fixed < TC_SMEM_MAX ? (int)((TC_SMEM_MAX - fixed) / L.chunk_bytes) : 0;
-  if (nstage > nck_max) nstage = nck_max < 3 ? 3 : nck_max;
+  const int want = nck_max < 3 ? 3 : nck_max;  // a tile-step of chunks, at least three
+  if (nstage > want) nstage = want;
   if (nstage > TW_MAX_STAGES) nstage = TW_MAX_STAGES;
   if (nstage < nck_max) nstage = nstage / TW_NCONV * TW_NCONV;
   L.NS = nstage;
@@ -170,7 +171,7 @@ bool tcw_supported(int n, int D, int A, int H, int prec) {
   if (D < 1 || D > 256 || D % 8 != 0 || n < 4 || n > 32 || A < 1 || A > TW_NQ) return false;
   if ((n * A) % 16 != 0) return false;  // an environment's availability bytes are bulk-copied and stored as 16-byte pieces
   const TwLayout L = tw_layout(n, D, A, rec_bytes_of(n, D, A));
-  return L.ept >= TW_G && L.NS >= 3 && L.NW >= 2 && L.n_slices <= TW_MAX_SLICES && L.total <= TC_SMEM_MAX;
+  return L.ept >= TW_G && L.NS >= 2 && L.NW >= 2 && L.n_slices <= TW_MAX_SLICES && L.total <= TC_SMEM_MAX;
 }
 
 size_t tcw_wpack_bytes(int n, int D, int A) {

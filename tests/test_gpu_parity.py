@@ -504,7 +504,7 @@ def test_streamed_hidden128_kernel_shapes_episode_ends_and_split_launches():
     chunks, one tile, more tiles than blocks, agent counts that do not divide 128, observation widths that need padding
     to the MMA's K step; an episode end in every step and never; launches of one step and split rollouts."""
     for over in (dict(E=130, n=8, D=80, A=14, C=260), dict(E=1, n=4, A=4, D=8, C=2), dict(E=37, n=16, A=5, D=16, C=74),
-                 dict(E=9, n=32, A=2, D=40, C=9), dict(E=2500, n=8, A=6, D=72, C=2500), dict(E=333, n=12, A=4, D=88, C=333)):
+                 dict(E=9, n=32, A=2, D=40, C=9), dict(E=2500, n=8, A=6, D=72, C=2500), dict(E=333, n=12, A=12, D=56, C=333)):
         cfg = workloads.small_config(H=128, L=7, T=20, precision="bf16", **over)
         w = workloads.make_weights(cfg)
         actor, acts, q = run_gpu_rollout(cfg, w, kernel="pipelined", splits=[1, 6, 13])
