@@ -55,14 +55,15 @@ extern "C" {
                               * wherever the shape is supported, at every batch size; otherwise, and for fp32, FFMA */
 #define MARL_KERNEL_FFMA 1   /* CUDA-core kernel: any shape, both precisions */
 #define MARL_KERNEL_TENSOR 2 /* one-tile tcgen05 kernel: bf16 only; create fails if the shape is unsupported */
-#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, at least 4 agents; hidden 64 with n_agents * n_actions
-                                        * a multiple of 4, or hidden 128 with at most 16 actions, obs_dim a multiple of
-                                        * 8 and n_agents * n_actions a multiple of 16 (weights streamed from L2, dense
-                                        * launches only); create fails otherwise.  Inputs that are not 16-byte
-                                        * aligned (or, where an environment's observation or availability block is
-                                        * not a 16-byte multiple, an environment count that is not a multiple of 4)
-                                        * fall back, per call, to the one-tile kernel where the shape allows it,
-                                        * else to the FFMA kernel */
+#define MARL_KERNEL_TENSOR_PIPELINED 3 /* pipelined tcgen05 kernel: bf16, at least 4 agents; hidden 64, or hidden 128
+                                        * with at most 16 actions, obs_dim a multiple of 8 and n_agents * n_actions a
+                                        * multiple of 16 (weights streamed from L2, dense launches only); create
+                                        * fails otherwise.  Inputs that are not 16-byte aligned fall back, per call,
+                                        * to the one-tile kernel where the shape allows it, else to the FFMA kernel;
+                                        * so do calls whose availability block (batch * n_agents * n_actions bytes)
+                                        * is not a 16-byte multiple when an environment's is not, and calls with an
+                                        * environment count that is not a multiple of 4 when obs_dim is not a
+                                        * multiple of 8 */
 
 #define MARL_MAX_AGENT_TYPES 4
 

@@ -69,7 +69,8 @@ struct TpBars {
   uint32_t tmem_base, abort;
 };
 
-static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
+// M, sms: the launch's batch and the number of blocks it may use (0: the largest tiles, for the shape check).
+static TpLayout tp_layout(int n, int D, int A, int rec_bytes, int M = 0, int sms = 0) {
   const TcLayout W = tc_layout(n, D, A, rec_bytes);
   TpLayout L;
   memset(&L, 0, sizeof(L));
@@ -79,13 +80,29 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.obs_bytes = (uint32_t)(n * D) * 4u;
   L.av_bytes = (uint32_t)(n * A);
   L.prefix_bytes = L.obs_bytes + L.av_bytes;  // of one environment in staging: [obs of the chunk | avail of the chunk]
-  // Shapes whose per-environment blocks are not 16-byte multiples ("plain"): whole chunks still are (4 n D floats,
-  // 4 n A bytes with n A a multiple of 4), so they load the same way, in tiles of whole chunks; the converters then
-  // read and store observations word by word instead of the store warp's bulk stores.
-  L.plain = (D % 8 != 0 || (n * A) % 16 != 0) ? 1 : 0;
-  if (L.plain) L.ept = L.ept / TP_G * TP_G;
+  // Shapes whose per-environment blocks are not 16-byte multiples ("plain"): a whole chunk's observations still are
+  // (4 n D floats), so they load the same way, in tiles of whole chunks; the converters then lay observations and
+  // availability bytes out as the records want them, for the store warp's bulk stores.
+  // plain = 1: observation rows that are not 16-byte multiples (word-by-word path, tiles of whole chunks so that
+  // every chunk starts on a 16-byte boundary); plain = 2: only the availability blocks are unaligned - observations
+  // take the aligned path, availability bytes the shifted one.
+  L.plain = D % 8 != 0 ? 1 : ((n * A) % 16 != 0 ? 2 : 0);
+  if (L.plain == 1) L.ept = L.ept / TP_G * TP_G;
+  // The plain shapes are bound by their converters, whose work grows with the tile: the smallest tile that keeps the
+  // number of waves evens the blocks out (4096 environments of 5 agents: 164 tiles of 25 on 148 blocks take two
+  // waves, and so do 293 tiles of 14, each at half the conversion).  The aligned shapes run at the step's dependency
+  // chain whatever the tile holds, so they keep full tiles.
+  if (L.plain != 0 && M > 0 && sms > 0) {
+    const int tiles = (M + L.ept - 1) / L.ept, waves = (tiles + sms - 1) / sms;
+    int e2 = (M + waves * sms - 1) / (waves * sms);
+    if (L.plain == 1) e2 = (e2 + TP_G - 1) / TP_G * TP_G;
+    if (e2 < TP_G) e2 = TP_G;
+    if (e2 < L.ept) L.ept = e2;
+  }
   L.tail_bytes = (uint32_t)rec_bytes - (up16(L.obs_bytes) + up16(L.av_bytes));
-  L.chunk_bytes = TP_G * L.prefix_bytes;
+  // (plain shapes: a chunk's availability bytes need not start on a 16-byte boundary of the input array; the load
+  // then covers the aligned range around them, at most 30 bytes more)
+  L.chunk_bytes = L.plain ? TP_G * L.obs_bytes + up16(TP_G * L.av_bytes) + 16u : TP_G * L.prefix_bytes;
   uint32_t o = L.wbytes;
   L.off_x = o; o += up16((uint32_t)L.nchunk * TC_LBO_X);
   L.off_y = o; o += 8 * TC_LBO_A;
@@ -103,9 +120,9 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   L.off_stage = o;
   // plain shapes: the converters also lay observations and availability bytes out as the records want them (each
   // block padded to 16 bytes), one image per staging slot, for the store warp's bulk stores
-  L.rs_env = L.plain ? up16(L.obs_bytes) + up16(L.av_bytes) : 0;  // the record's prefix [obs | avail], padded as in the ring
+  L.rs_env = L.plain == 1 ? up16(L.obs_bytes) + up16(L.av_bytes) : 0;  // the record's prefix [obs | avail], padded as in the ring
   L.rs_bytes = TP_G * L.rs_env;
-  const uint32_t room = o + 32 < TC_SMEM_MAX ? TC_SMEM_MAX - o - 32 : 0;
+  const uint32_t room = o + 64 < TC_SMEM_MAX ? TC_SMEM_MAX - o - 64 : 0;
   int ns = (int)(room / (L.chunk_bytes + L.rs_bytes));
   if (ns > TP_MAX_STAGES) ns = TP_MAX_STAGES;
   if (ns < 0) ns = 0;
@@ -116,17 +133,16 @@ static TpLayout tp_layout(int n, int D, int A, int rec_bytes) {
   const int nck_max = (L.ept + TP_G - 1) / TP_G;
   if (ns < nck_max) ns = ns / (TP_CONV / 32) * (TP_CONV / 32);
   L.NS = ns;
-  L.off_rstage = o + (uint32_t)ns * L.chunk_bytes + 32;  // (+32: the mask words read a few bytes past a row)
+  L.off_rstage = o + (uint32_t)ns * L.chunk_bytes + 64;  // (+64: the mask words read a few bytes past a row)
   L.total = L.off_rstage + (uint32_t)ns * L.rs_bytes;
   return L;
 }
 
-// Shapes this kernel takes: at least 4 agents (tiles of at most 32 environments, one lane each) and chunks of
-// four environments whose observation and availability blocks are 16-byte multiples.
+// Shapes this kernel takes: at least 4 agents (tiles of at most 32 environments, one lane each) and a staging ring
+// of at least three chunks of four environments.
 bool tcp_supported(int n, int D, int A, int H, int prec) {
   if (prec != MARL_PRECISION_BF16 || H != TC_H) return false;
   if (D < 1 || D > 256 || n < 4 || n > 32 || A < 1 || A > 32) return false;
-  if ((n * A) % 4 != 0) return false;  // a chunk's availability bytes must be a 16-byte multiple
   const TpLayout L = tp_layout(n, D, A, rec_bytes_of(n, D, A));
   // enough staging for loads to run ahead of the network (tp_layout leaves 0 where the ring would be unsafe)
   return L.ept >= TP_G && L.NS >= 3 && L.total <= TC_SMEM_MAX;
@@ -191,7 +207,8 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
   __syncwarp();
 }
 
-// PLAIN: the word-by-word path of shapes whose per-environment blocks are not 16-byte multiples.
+// PM (TpLayout::plain) 1: the word-by-word path of shapes whose observation rows are not 16-byte multiples; 1 and 2:
+// availability blocks that may start anywhere inside a 16-byte unit of the input array.
 // MODE 1, 2 (LIST): the call's rows are the environments of p.env_ids (a partial step); inputs, the last step's
 // actions and the tiling follow the row, state, ring cursors, the draw's key and the trace follow the environment.
 // MODE 2 (LAG, one step per launch): reward/done are the outcome of each environment's previous action: they complete
@@ -200,7 +217,7 @@ __device__ __forceinline__ void tp_issue_hside(const TpLayout& L, uint32_t sb, u
 // hidden-state rows then move coalesced through a scratch and the next tile's rows are prefetched into L2 (modes 1
 // and 2 do the same).  Launches of many steps keep the shorter transition code: its footprint in the step loop's
 // instruction stream and registers costs them more (1.2 %) than the transition saves.
-template <int NQ, bool PLAIN, int MODE>
+template <int NQ, int PM, int MODE>
 __global__ void __launch_bounds__(TP_THREADS, 1)
     actor_tcp_kernel(const __grid_constant__ ActorParams p, const __grid_constant__ TpLayout L) {
   constexpr bool LIST = MODE == 1 || MODE == 2, LAG = MODE == 2, FASTX = MODE != 0;
@@ -409,16 +426,19 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
               mbar_wait(&B->cfree[qslot], qpar, abortf);
               mbar_wait(&B->sfree[qslot], qpar, abortf);
             }
-            if (lane == 0) mbar_arrive_expect_tx(&B->full[qslot], (uint32_t)ge * L.prefix_bytes);
-            __syncwarp();
             const size_t env0 = (size_t)tile * L.ept + (size_t)(c * TP_G);
+            // availability bytes of the chunk: [a0, a0 + ge n A) of the input array; plain shapes load the 16-byte
+            // aligned range around them (inside the array: the launcher checks that the step's block ends aligned)
+            const size_t a0 = (size_t)s * p.avail_step_stride + env0 * (size_t)(n * A);
+            const size_t b0 = PM != 0 ? a0 & ~(size_t)15 : a0;
+            const uint32_t av_load = PM != 0 ? (uint32_t)(((a0 + (size_t)ge * L.av_bytes + 15) & ~(size_t)15) - b0) : (uint32_t)ge * L.av_bytes;
+            if (lane == 0) mbar_arrive_expect_tx(&B->full[qslot], (uint32_t)ge * L.obs_bytes + av_load);
+            __syncwarp();
             uint8_t* dst = stage + qslot * L.chunk_bytes;
             if (lane == 0)
               bulk_load(dst, p.obs + (size_t)s * p.obs_step_stride + env0 * (size_t)(n * D), (uint32_t)ge * L.obs_bytes,
                         &B->full[qslot]);
-            if (lane == 1)
-              bulk_load(dst + TP_G * L.obs_bytes, p.avail + (size_t)s * p.avail_step_stride + env0 * (size_t)(n * A),
-                        (uint32_t)ge * L.av_bytes, &B->full[qslot]);
+            if (lane == 1) bulk_load(dst + TP_G * L.obs_bytes, p.avail + b0, av_load, &B->full[qslot]);
             ++q;
             if (++qslot == (uint32_t)NS) {
               qslot = 0;
@@ -544,12 +564,12 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           for (int c = 0; c < nck; ++c) {
             const int ge = min(TP_G, ne - c * TP_G);
             // plain shapes: the image the converters wrote, once they are done with the chunk; else the staged block
-            mbar_wait(PLAIN ? &B->cfree[qslot] : &B->full[qslot], qpar, abortf);
+            mbar_wait(PM == 1 ? &B->cfree[qslot] : &B->full[qslot], qpar, abortf);
             if (lane < ge) {
               const unsigned long long rec = dstp_s[(kstep & (TP_DST_DEPTH - 1)) * 32 + c * TP_G + lane];
-              const uint8_t* from = PLAIN ? smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)lane * L.rs_env
+              const uint8_t* from = PM == 1 ? smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)lane * L.rs_env
                                             : stage + qslot * L.chunk_bytes + (uint32_t)lane * L.obs_bytes;
-              if (rec) bulk_store(reinterpret_cast<void*>(rec), from, PLAIN ? L.rs_env : L.obs_bytes);
+              if (rec) bulk_store(reinterpret_cast<void*>(rec), from, PM == 1 ? L.rs_env : L.obs_bytes);
             }
             bulk_commit();
             // every lane commits one (possibly empty) group per chunk, so "all but the latest" covers chunk q - 1
@@ -576,6 +596,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
     // Each of the four warps takes whole chunks (chunk c of a step goes to warp c % 4), so a step's chunks are
     // converted side by side; thread ci then owns row ci of the tile for the epsilon draw.
     const int ci = tid - 256, cw = warp - 8;
+    const int li = lane, ls = 32;
     const uint32_t inv_nchunk = 0xFFFFFFFFu / (uint32_t)L.nchunk + 1u;  // j / nchunk == umulhi(j, inv) for j < 2^16
     const uint32_t amask = A >= 32 ? 0xFFFFFFFFu : ((1u << A) - 1u);
     uint32_t it = 0, qbase = 0;  // steps and chunks before this step
@@ -598,22 +619,39 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           const unsigned long long* recs = dstp_s + (it & (TP_DST_DEPTH - 1)) * 32 + c * TP_G;  // this chunk's records
           mbar_wait(&B->full[qslot], qpar, abortf);
           const int items = Rc * L.nchunk;
-          if (PLAIN) {
-            // rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record image
-            for (int j = lane; j < items; j += 32) {
-              const int rr = (int)__umulhi((uint32_t)j, inv_nchunk), cc = j - rr * L.nchunk;
-              const int envc = rowenv_s[rr];
-              const float* srow = reinterpret_cast<const float*>(src) + rr * D;
-              float* drow = reinterpret_cast<float*>(smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)envc * L.rs_env) + (rr - envc * n) * D;
-              float v[8];
+          if (PM == 1) {
+            // Rows are not 16-byte aligned: word by word, eight columns per item, to the operand and to the record
+            // image.  Consecutive lanes take consecutive ROWS of one column group: a row stride of D words is odd for
+            // most such shapes, so the lanes' words fall in different banks (lanes eight words apart would share four).
+            const uint32_t inv_Rc = 0xFFFFFFFFu / (uint32_t)Rc + 1u;  // j / Rc == umulhi(j, inv) for j < 2^16
+            for (int j = lane; j < items; j += 64) {  // two items per thread and pass: sixteen loads in flight
+              float v[2][8];
+              int cc[2], rr[2];
+              bool on[2];
+              float* drow[2];
 #pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const int col = cc * 8 + k;
-                v[k] = col < D ? srow[col] : 0.f;
-                if (col < D) drow[col] = v[k];
+              for (int u = 0; u < 2; ++u) {
+                const int jj = j + 32 * u;
+                on[u] = jj < items;
+                cc[u] = on[u] ? (int)__umulhi((uint32_t)jj, inv_Rc) : 0;
+                rr[u] = on[u] ? jj - cc[u] * Rc : 0;
+                const int envc = rowenv_s[rr[u]];
+                const float* srow = reinterpret_cast<const float*>(src) + rr[u] * D;
+                drow[u] = reinterpret_cast<float*>(smem + L.off_rstage + qslot * L.rs_bytes + (uint32_t)envc * L.rs_env) + (rr[u] - envc * n) * D;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[u][k] = (on[u] && cc[u] * 8 + k < D) ? srow[cc[u] * 8 + k] : 0.f;
               }
-              *reinterpret_cast<uint4*>(xb + (uint32_t)cc * TC_LBO_X + (uint32_t)(r0 + rr) * 16u) =
-                  make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {  // (stores after all the loads: a store between them would order them one by one)
+                if (on[u]) {
+#pragma unroll
+                  for (int k = 0; k < 8; ++k)
+                    if (cc[u] * 8 + k < D) drow[u][cc[u] * 8 + k] = v[u][k];
+                  *reinterpret_cast<uint4*>(xb + (uint32_t)cc[u] * TC_LBO_X + (uint32_t)(r0 + rr[u]) * 16u) =
+                      make_uint4(pack_bf16x2(v[u][0], v[u][1]), pack_bf16x2(v[u][2], v[u][3]), pack_bf16x2(v[u][4], v[u][5]),
+                                 pack_bf16x2(v[u][6], v[u][7]));
+                }
+              }
             }
           } else
           for (int j = lane; j < items; j += 64) {
@@ -643,14 +681,29 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
               }
             }
           }
-          const uint8_t* avs = src + TP_G * L.obs_bytes;  // the chunk's availability bytes, rows contiguous
-          if (PLAIN) {
-            const uint32_t per_env = L.av_bytes / 4u;  // n A is a multiple of 4
+          // the chunk's availability bytes, rows contiguous; plain shapes: from byte `shift` of the loaded range
+          const uint8_t* avs = src + TP_G * L.obs_bytes;
+          const uint32_t shift = PM != 0 ? (uint32_t)(((size_t)(e0 + c * TP_G) * (size_t)(n * A)) & 15u) : 0u;
+          if (PM != 0) {
+            // To the record images (1) or straight to the records (2): word j of an environment's block is put
+            // together from the two loaded words that hold its bytes; bytes beyond the block stay zero (padding of
+            // the record).
+            const uint32_t per_env = (L.av_bytes + 3u) / 4u;
             const uint32_t inv = 0xFFFFFFFFu / per_env + 1u;  // idx / per_env == umulhi(idx, inv) for idx < 2^16
             uint8_t* img = smem + L.off_rstage + qslot * L.rs_bytes + p.rl.off_avail;
-            for (uint32_t i = lane; i < (uint32_t)ge * per_env; i += 32) {
-              const uint32_t envc = __umulhi(i, inv);
-              reinterpret_cast<uint32_t*>(img + envc * L.rs_env)[i - envc * per_env] = reinterpret_cast<const uint32_t*>(avs)[i];
+            for (uint32_t i = li; i < (uint32_t)ge * per_env; i += ls) {
+              const uint32_t envc = __umulhi(i, inv), j = i - envc * per_env;
+              const uint32_t sb = shift + envc * L.av_bytes + 4u * j;  // first source byte of the word
+              const uint32_t* w = reinterpret_cast<const uint32_t*>(avs + (sb & ~3u));
+              uint32_t v = __funnelshift_r(w[0], w[1], 8u * (sb & 3u));
+              const uint32_t left = L.av_bytes - 4u * j;  // bytes of the block from this word on
+              if (left < 4u) v &= (1u << (8u * left)) - 1u;
+              if (PM == 1) {
+                reinterpret_cast<uint32_t*>(img + envc * L.rs_env)[j] = v;
+              } else {
+                const unsigned long long rec = recs[envc];
+                if (rec) reinterpret_cast<uint32_t*>(rec + p.rl.off_avail)[j] = v;
+              }
             }
           } else {
             const uint32_t per_env = L.av_bytes / 16u;
@@ -663,8 +716,8 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
           // Availability masks of the chunk's rows.  A row's A bytes are read as aligned words (a few bytes beyond
           // the row are read and masked off) and each word's four "byte is non-zero" flags are gathered with one
           // multiply: short code, few loads.
-          for (int rc = lane; rc < Rc; rc += 32) {
-            const uint32_t off = (uint32_t)(rc * A);
+          for (int rc = li; rc < Rc; rc += ls) {
+            const uint32_t off = shift + (uint32_t)(rc * A);
             const uint32_t* w = reinterpret_cast<const uint32_t*>(avs + (off & ~3u));
             unsigned long long bits = 0;
 #pragma unroll
@@ -675,7 +728,7 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
             }
             sel[r0 + rc].x = (uint32_t)(bits >> (off & 3u)) & amask;
           }
-          if (PLAIN) fence_proxy_async_smem();  // the record image is read by the store warp's bulk stores
+          if (PM == 1) fence_proxy_async_smem();  // the record image is read by the store warp's bulk stores
           __syncwarp();
           if (lane == 0) mbar_arrive(&B->cfree[qslot]);
         }
@@ -1025,27 +1078,32 @@ __global__ void __launch_bounds__(TP_THREADS, 1)
 // Returns the number of kernels launched, 0 if this launch's pointers do not meet the kernel's alignment
 // needs (the caller then uses the one-tile kernel), or a negative cudaError.
 int launch_actor_tcp(const ActorParams& p_in, int sms, cudaStream_t stream) {
-  const TpLayout L = tp_layout(p_in.n, p_in.D, p_in.A, (int)p_in.rl.rec_bytes);
+  const TpLayout L = tp_layout(p_in.n, p_in.D, p_in.A, (int)p_in.rl.rec_bytes, p_in.M, sms);
   ActorParams p = p_in;
   p.ept = L.ept;  // (tiles of whole chunks for the plain shapes)
   p.num_tiles = (p.M + L.ept - 1) / L.ept;
   if (reinterpret_cast<uintptr_t>(p.obs) % 16 || reinterpret_cast<uintptr_t>(p.avail) % 16) return 0;
   if ((p.obs_step_stride * 4) % 16 || p.avail_step_stride % 16) return 0;
-  if (L.plain && p.M % TP_G != 0) return 0;  // a last chunk of fewer environments would not be a 16-byte multiple
+  // plain shapes: a last chunk of fewer environments would not be a 16-byte multiple, and the aligned range around
+  // the last chunk's availability bytes must end inside the step's block
+  if (L.plain == 1 && p.M % TP_G != 0) return 0;
+  if (L.plain != 0 && ((size_t)p.M * p.n * p.A) % 16 != 0) return 0;
   const int mode = p.env_ids == nullptr ? (p.T < 8 ? 3 : 0) : (p.lagged ? 2 : 1);
   if (p.lagged && (mode != 2 || p.T != 1)) return 0;  // late outcomes: one step per launch over a list
   auto pick = [&](auto nq) {
     constexpr int Q = decltype(nq)::value;
-    return mode == 3 ? (L.plain ? actor_tcp_kernel<Q, true, 3> : actor_tcp_kernel<Q, false, 3>)
-         : mode == 2 ? (L.plain ? actor_tcp_kernel<Q, true, 2> : actor_tcp_kernel<Q, false, 2>)
-         : mode == 1 ? (L.plain ? actor_tcp_kernel<Q, true, 1> : actor_tcp_kernel<Q, false, 1>)
-                     : (L.plain ? actor_tcp_kernel<Q, true, 0> : actor_tcp_kernel<Q, false, 0>);
+    auto of_mode = [&](auto md) {
+      constexpr int MD = decltype(md)::value;
+      return L.plain == 1 ? actor_tcp_kernel<Q, 1, MD> : L.plain == 2 ? actor_tcp_kernel<Q, 2, MD> : actor_tcp_kernel<Q, 0, MD>;
+    };
+    return mode == 3 ? of_mode(std::integral_constant<int, 3>()) : mode == 2 ? of_mode(std::integral_constant<int, 2>())
+         : mode == 1 ? of_mode(std::integral_constant<int, 1>()) : of_mode(std::integral_constant<int, 0>());
   };
   auto kernel = L.NQ == 16 ? pick(std::integral_constant<int, 16>()) : pick(std::integral_constant<int, 32>());
-  static uint32_t configured[16][SMEM_OPTIN_DEVICES];
+  static uint32_t configured[24][SMEM_OPTIN_DEVICES];
   {
     const cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L.total,
-                                              configured[(L.NQ == 16 ? 0 : 1) + (L.plain ? 2 : 0) + 4 * mode]);
+                                              configured[(L.NQ == 16 ? 0 : 1) + 2 * L.plain + 6 * mode]);
     if (e != cudaSuccess) return -(int)e;
   }
   int grid = p.num_tiles < sms ? p.num_tiles : sms;

@@ -430,16 +430,14 @@ def test_pipelined_kernel_falls_back_on_unaligned_inputs():
 
 @pytest.mark.parametrize("seed", range(4))
 def test_pipelined_kernel_seeded_shapes(seed):
-    """Seeded shapes inside the pipelined kernel's stated domain (4..32 agents, 1..32 actions with n * A a multiple of
-    four, 1..256 observation features): environment counts that leave ragged tiles and partial chunks, short and
-    long slots, single-step and multi-step launches mixed.  Each is refereed against the oracle on every row."""
+    """Seeded shapes inside the pipelined kernel's stated domain (4..32 agents, 1..32 actions, 1..256 observation
+    features; n * A odd or even): environment counts that leave ragged tiles and partial chunks, short and long
+    slots, single-step and multi-step launches mixed.  Each is refereed against the oracle on every row."""
     rng = np.random.default_rng(1000 + seed)
     done_shapes = 0
-    while done_shapes < 4:
+    while done_shapes < 5:
         n = int(rng.integers(4, 33))
         A = int(rng.integers(1, 33))
-        if (n * A) % 4:
-            continue
         D = int(rng.integers(1, 257))
         tile_envs = max(1, 128 // n)
         E = int(rng.integers(1, 4 * tile_envs + 3))
@@ -463,6 +461,27 @@ def test_pipelined_kernel_seeded_shapes(seed):
         print(f"   {res}")
         actor.destroy()
         done_shapes += 1
+
+
+def test_pipelined_kernel_shapes_whose_availability_rows_are_not_word_aligned():
+    """n * A not a multiple of four (workload 3's 5 x 11 among them): a chunk's availability bytes start anywhere
+    inside a 16-byte unit of the input array; the kernel loads the aligned range around them and shifts.  The
+    environment counts are multiples of 16, so every launch stays on the pipelined kernel: decisions, records and
+    state equal the one-tile kernel's (where that kernel takes the shape), and every row passes the referee."""
+    for over in (dict(n=5, A=11, D=80, E=208), dict(n=7, A=9, D=33, E=112), dict(n=5, A=11, D=55, E=64),
+                 dict(n=9, A=3, D=16, E=48), dict(n=13, A=17, D=24, E=32)):
+        cfg = workloads.small_config(H=64, precision="bf16", C=2 * over["E"], L=5, T=12,
+                                     env=dict(done_thresh24=1 << 21), **over)
+        w = workloads.make_weights(cfg)
+        a, acts_a, q_a = run_gpu_rollout(cfg, w, kernel="pipelined", splits=[7, 1, 4])
+        assert a.kernel_name == "tcgen05-pipelined"
+        if over["D"] % 8 == 0:  # (the one-tile kernel takes observation rows of whole 8-column groups only)
+            b, acts_b, q_b = run_gpu_rollout(cfg, w, kernel="tensor", splits=[7, 1, 4])
+            assert b.kernel_name == "tcgen05"
+            _assert_same_rollout(a, acts_a, q_a, b, acts_b, q_b, tag=str(over))
+            b.destroy()
+        print(over, referee(cfg, w, a, acts_a, q_a))
+        a.destroy()
 
 
 def test_shape_with_a_short_staging_ring_leaves_the_pipelined_kernel():
