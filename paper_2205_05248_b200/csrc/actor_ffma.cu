@@ -5,13 +5,13 @@
 // hidden state per environment and agent), so the hidden state, the last actions and the ring cursors of
 // the tile stay in shared memory for the whole launch.  Per step the block runs the worker's decision
 // (Algorithm 2: observations in, policy network, actions out) and the actor's recording of the step
-// (Algorithm 1), in six phases separated by block barriers:
-//   A  stage obs (-> shared, and verbatim into the ring record), availability masks, open slot headers
+// (Algorithm 1), in phases separated by block barriers:
+//   A  stage obs (-> shared, and verbatim into the ring record), availability masks, open slot headers; a second set
+//      of threads makes the epsilon draws, which need only the availability bytes
 //   B  fc1 + one-hot column gathers + ReLU                       (register-tiled 4 rows x 4 columns)
 //   C  GRU cell: both gate GEMMs, gate math, new hidden state    (same tiling, 64 accumulators)
-//   D  fc2
-//   E  masked greedy choice, epsilon draw, ring/trace writes     (one thread per row)
-//   F  reward/done, episode bookkeeping, hidden-state reset      (one thread per environment)
+//   D  fc2, masked greedy choice, ring/trace writes              (four threads per row, Q in registers)
+//   F  reward/done, episode bookkeeping, hidden-state reset      (one thread per environment, then a warp per row)
 // Weights are read through the read-only path from k-major copies, so a warp's load of four output
 // columns for one k is one contiguous 256-byte segment.
 #include "common.cuh"
@@ -21,18 +21,17 @@ namespace marl {
 
 constexpr int FF_RMAX = 64;      // rows per tile
 constexpr int FF_THREADS = 256;
-constexpr int FF_QSTRIDE = 33;   // row stride of the Q tile (odd: one row per thread without conflicts)
 constexpr int FF_PRE = 8;        // float4 registers per thread that hold the next step's observations
 
 struct FfmaSmem {
   int Dp, Hp, wsmem;
-  size_t off_xs, off_ys, off_hs, off_qs, off_mask, off_la, off_env, off_w, w_floats, total;
+  size_t off_xs, off_ys, off_hs, off_pick, off_mask, off_la, off_env, off_w, w_floats, total;
 };
 
 // Floats of the weight image kept in shared memory when it fits (hidden size 64): the k-major matrices
-// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2 [A][H], in this order.
+// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2T [H][A rounded up to 4], in this order.
 __host__ __device__ inline size_t ffma_weight_floats(int n, int D, int A, int H) {
-  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)A * H;
+  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)((A + 3) & ~3) * H;
 }
 
 __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H) {
@@ -45,7 +44,7 @@ __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H)
   s.off_xs = o; o += sizeof(float) * FF_RMAX * s.Dp;
   s.off_ys = o; o += sizeof(float) * FF_RMAX * s.Hp;
   s.off_hs = o; o += sizeof(float) * 2 * FF_RMAX * s.Hp;
-  s.off_qs = o; o += sizeof(float) * FF_RMAX * FF_QSTRIDE;
+  s.off_pick = o; o += sizeof(int32_t) * FF_RMAX;
   s.off_mask = o; o += sizeof(uint32_t) * FF_RMAX;
   s.off_la = o; o += sizeof(int32_t) * FF_RMAX;
   s.off_env = o; o += 40 * FF_RMAX;  // per-environment scratch: see EnvSlot
@@ -101,7 +100,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   float* xs = reinterpret_cast<float*>(smem + sl.off_xs);
   float* ys = reinterpret_cast<float*>(smem + sl.off_ys);
   float* hs = reinterpret_cast<float*>(smem + sl.off_hs);
-  float* qs = reinterpret_cast<float*>(smem + sl.off_qs);
+  int32_t* picks = reinterpret_cast<int32_t*>(smem + sl.off_pick);  // the epsilon draw of every row: a random action or -1
   uint32_t* masks = reinterpret_cast<uint32_t*>(smem + sl.off_mask);
   int32_t* la = reinterpret_cast<int32_t*>(smem + sl.off_la);
   EnvSlot* envs = reinterpret_cast<EnvSlot*>(smem + sl.off_env);
@@ -129,7 +128,12 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
     const size_t n1 = (size_t)(p.I + 4) * H, n2 = (size_t)H * H3, n3 = (size_t)A * H;
     for (size_t i = tid; i < n1; i += FF_THREADS) wsm[i] = p.W1T[i];
     for (size_t i = tid; i < n2; i += FF_THREADS) { wsm[n1 + i] = p.WihT[i]; wsm[n1 + n2 + i] = p.WhhT[i]; }
-    for (size_t i = tid; i < n3; i += FF_THREADS) wsm[n1 + 2 * n2 + i] = p.W2[i];
+    const int AQ = (A + 3) & ~3;  // W2 transposed: the actions of one k side by side, padded with zeros
+    for (size_t i = tid; i < (size_t)AQ * H; i += FF_THREADS) {
+      const int k = (int)(i / AQ), a = (int)(i - (size_t)k * AQ);
+      wsm[n1 + 2 * n2 + i] = a < A ? p.W2[(size_t)a * H + k] : 0.f;
+    }
+    (void)n3;
     W1T = wsm; WihT = wsm + n1; WhhT = wsm + n1 + n2; W2 = wsm + n1 + 2 * n2;
   }
   __syncthreads();
@@ -261,6 +265,16 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             if (es.ok) dst[a] = b;
           }
           masks[tid] = m;
+        }
+        if (tid >= FF_RMAX && tid < FF_RMAX + R) {
+          // The epsilon draw needs only the availability bytes (Algorithm 2 draws before it looks at Q): a second
+          // set of threads reads them again and draws while the first set records them.
+          const int r = tid - FF_RMAX, el = r / n, ai = r - el * n;
+          const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + ((size_t)e0 * n + r) * A;
+          uint32_t m = 0;
+          for (int a = 0; a < A; ++a)
+            if (av[a]) m |= 1u << a;
+          picks[r] = m ? draw_explore(m, eps, p.seed, t, (uint32_t)envs[el].eid, (uint32_t)ai) : -1;
         }
         if (tid < ne) {
           EnvSlot& es = envs[tid];
@@ -401,66 +415,115 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       }
       __syncthreads();
 
-      // ---- phase D: fc2 (four threads per row, actions striped over them) ----
+      // ---- phase D: fc2, masked greedy choice and recording: four threads per row, each with the Q values of
+      //      actions 4 part .. 4 part + 3 and 16 + 4 part .. 16 + 4 part + 3 in registers; the row's maximum and the
+      //      set of near-maximal actions go round the four lanes by shuffles ----
       {
         const int r = tid >> 2, part = tid & 3;
+        const bool live = r < R;
         const size_t toff = row_type(r) * tstride;  // this row's own network
-        float acc[8];
+        float q[2][4];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          const int a = part + 4 * m;
-          acc[m] = a < A ? __ldg(p.b2 + toff + a) : 0.f;
-        }
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int a = 16 * g + 4 * part + c;
+            q[g][c] = a < A ? __ldg(p.b2 + toff + a) : 0.f;
+          }
         const float* hv = hs + nxt * hbuf + r * Hp;
-        for (int k = 0; k < H; k += 4) {
-          const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
+        if (WS) {
+          const int AQ = (A + 3) & ~3;
+          const float* wcol = W2 + 4 * part;  // W2T [k][AQ]
+          for (int k = 0; k < H; k += 4) {
+            const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
 #pragma unroll
-          for (int m = 0; m < 8; ++m) {
-            const int a = part + 4 * m;
-            if (a < A) {
-              const float4 w = wload4<WS>(W2 + toff + (size_t)a * H + k);
-              acc[m] = fmaf(v.x, w.x, acc[m]);
-              acc[m] = fmaf(v.y, w.y, acc[m]);
-              acc[m] = fmaf(v.z, w.z, acc[m]);
-              acc[m] = fmaf(v.w, w.w, acc[m]);
+            for (int kk = 0; kk < 4; ++kk) {
+              const float vk = kk == 0 ? v.x : kk == 1 ? v.y : kk == 2 ? v.z : v.w;
+#pragma unroll
+              for (int g = 0; g < 2; ++g) {
+                if (16 * g + 4 * part < A) {
+                  const float4 w = *reinterpret_cast<const float4*>(wcol + (size_t)(k + kk) * AQ + 16 * g);
+                  q[g][0] = fmaf(vk, w.x, q[g][0]); q[g][1] = fmaf(vk, w.y, q[g][1]);
+                  q[g][2] = fmaf(vk, w.z, q[g][2]); q[g][3] = fmaf(vk, w.w, q[g][3]);
+                }
+              }
             }
           }
-        }
+        } else {
+          for (int k = 0; k < H; k += 4) {
+            const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          const int a = part + 4 * m;
-          if (a < A) qs[r * FF_QSTRIDE + a] = acc[m];
+            for (int g = 0; g < 2; ++g)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const int a = 16 * g + 4 * part + c;
+                if (a < A) {
+                  const float4 w = wload4<WS>(W2 + toff + (size_t)a * H + k);
+                  q[g][c] = fmaf(v.x, w.x, q[g][c]);
+                  q[g][c] = fmaf(v.y, w.y, q[g][c]);
+                  q[g][c] = fmaf(v.z, w.z, q[g][c]);
+                  q[g][c] = fmaf(v.w, w.w, q[g][c]);
+                }
+              }
+          }
         }
-      }
-      __syncthreads();
-
-      // ---- phase E: choice and recording, one thread per row ----
-      if (tid < R) {
-        const int el = tid / n, ai = tid - el * n;
-        const int e = envs[el].eid;
-        const float* qrow = qs + tid * FF_QSTRIDE;
-        uint32_t flags;
-        const int act = select_action([&](int a) { return qrow[a]; }, A, masks[tid], eps, p.seed, t,
-                                      (uint32_t)e, (uint32_t)ai, flags);
-        c_steps += 1;
-        c_explore += flags & 1u;
-        if (flags & 2u) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
-        la[tid] = act;
-        const EnvSlot& es = envs[el];
-        if (es.ok) {
+        // greedy rule: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr (a NaN never
+        // compares greater or equal and fmaxf ignores it, like the "greater than" scan of select_action)
+        const uint32_t mask = live ? masks[r] : 0u;
+        float m = -INFINITY;
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int a = 16 * g + 4 * part + c;
+            if (a < A && ((mask >> a) & 1u)) m = fmaxf(m, q[g][c]);
+          }
+        m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+        const float thr = __fsub_rn(m, 1e-4f);
+        uint32_t ge = 0;
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int a = 16 * g + 4 * part + c;
+            if (a < A && q[g][c] >= thr) ge |= 1u << a;
+          }
+        ge |= __shfl_xor_sync(0xFFFFFFFFu, ge, 1);
+        ge |= __shfl_xor_sync(0xFFFFFFFFu, ge, 2);
+        ge &= mask;
+        if (live) {
+          const int el = r / n, ai = r - el * n;
+          const int pick = picks[r];
+          const int greedy = ge ? __ffs(ge) - 1 : __ffs(mask) - 1;
+          const int act = mask == 0 ? 0 : (pick >= 0 ? pick : greedy);
+          const EnvSlot& es = envs[el];
+          const int e = es.eid;
           uint8_t* rec = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes;
-          float* qd = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
-          for (int a = 0; a < A; ++a) qd[a] = qrow[a];
-          reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
-        }
-        const int tk = p.trace_first + s;
-        if (tk < p.trace_cap) {
+          const int tk = p.trace_first + s;
           const size_t grow = ((size_t)tk * p.E + e) * n + ai;
-          if (p.trace_actions) p.trace_actions[grow] = act;
-          if (p.trace_q)
-            for (int a = 0; a < A; ++a) p.trace_q[grow * A + a] = qrow[a];
+          const bool traced = tk < p.trace_cap;
+          float* qd = reinterpret_cast<float*>(rec + p.rl.off_q) + ai * A;
+#pragma unroll
+          for (int g = 0; g < 2; ++g)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const int a = 16 * g + 4 * part + c;
+              if (a < A) {
+                if (es.ok) qd[a] = q[g][c];
+                if (traced && p.trace_q) p.trace_q[grow * A + a] = q[g][c];
+              }
+            }
+          if (part == 0) {
+            c_steps += 1;
+            c_explore += (mask != 0 && pick >= 0) ? 1u : 0u;
+            if (mask == 0) { c_noavail += 1; st_bits |= MARL_STATUS_NO_AVAIL; }
+            la[r] = act;
+            if (es.ok) reinterpret_cast<int32_t*>(rec + p.rl.off_action)[ai] = act;
+            if (traced && p.trace_actions) p.trace_actions[grow] = act;
+            if (p.actions_out && s == p.T - 1) p.actions_out[(size_t)(e0 + el) * n + ai] = act;
+          }
         }
-        if (p.actions_out && s == p.T - 1) p.actions_out[(size_t)(e0 + el) * n + ai] = act;
       }
       __syncthreads();  // the rows above read the cursors that the environment threads advance below
       // ---- phase F (first half): reward/done and the episode cursor, one thread per environment ----
@@ -487,12 +550,9 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       }
       __syncthreads();
       // ---- phase F (second half): a closed episode starts from a zero hidden state and no last action ----
-      for (int idx = tid; idx < R * H; idx += FF_THREADS) {
-        const int r = idx / H, j = idx - r * H;
-        if (envs[r / n].reset) {
-          hs[nxt * hbuf + r * Hp + j] = 0.f;
-        }
-      }
+      for (int r = tid >> 5; r < R; r += FF_THREADS / 32)  // a warp per row: the flag is read once, rows rarely reset
+        if (envs[r / n].reset)
+          for (int j = tid & 31; j < H; j += 32) hs[nxt * hbuf + r * Hp + j] = 0.f;
       if (tid < R && envs[tid / n].reset) la[tid] = -1;
       cur = nxt;
       __syncthreads();
