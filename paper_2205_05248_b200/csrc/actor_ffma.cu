@@ -14,6 +14,8 @@
 //   F  reward/done, episode bookkeeping, hidden-state reset      (one thread per environment, then a warp per row)
 // Weights are read through the read-only path from k-major copies, so a warp's load of four output
 // columns for one k is one contiguous 256-byte segment.
+#include <type_traits>
+
 #include "common.cuh"
 #include "launch_util.cuh"
 
@@ -29,9 +31,10 @@ struct FfmaSmem {
 };
 
 // Floats of the weight image kept in shared memory when it fits (hidden size 64): the k-major matrices
-// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2T [H][A rounded up to 4], in this order.
+// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2T [H][A rounded up to 4], then the biases b1 [H], b_ih [3H],
+// b_hh [3H] and b2 [A rounded up to 4], in this order.
 __host__ __device__ inline size_t ffma_weight_floats(int n, int D, int A, int H) {
-  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)((A + 3) & ~3) * H;
+  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)((A + 3) & ~3) * (H + 1) + 7 * (size_t)H;
 }
 
 __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H) {
@@ -75,6 +78,27 @@ template <bool WS>
 __device__ __forceinline__ float4 wload4(const float* ptr) {
   if (WS) return *reinterpret_cast<const float4*>(ptr);
   return __ldg(reinterpret_cast<const float4*>(ptr));
+}
+// Two fp32 values in one 64-bit register and the packed multiply-add on them (fma.rn.f32x2: each half is the IEEE
+// fused multiply-add of fmaf).  The FMA pipe does as many of them per clock as scalar ones would give - the peak is
+// the same - but a packed instruction takes one issue slot for two, which leaves slots for the loads of the GEMM loops.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// Four weights as two packed pairs.
+template <bool WS>
+__device__ __forceinline__ ulonglong2 wload22(const float* ptr) {
+  if (WS) return *reinterpret_cast<const ulonglong2*>(ptr);
+  return __ldg(reinterpret_cast<const ulonglong2*>(ptr));
 }
 // Volatile, so that the request stays where it is written: a whole step before the value is used.
 __device__ __forceinline__ float4 ldg_nc_v4(const float4* ptr) {
@@ -123,6 +147,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   for (int i = tid; i < (int)(sl.off_w / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;
   // weight pointers: the resident copy, or the k-major global arrays
   const float *W1T = p.W1T, *WihT = p.WihT, *WhhT = p.WhhT, *W2 = p.W2;
+  const float *B1 = p.b1, *BIH = p.bih, *BHH = p.bhh, *B2 = p.b2;  // (a phase that starts with a load from global memory waits for it every step)
   if (WS) {
     float* wsm = reinterpret_cast<float*>(smem + sl.off_w);
     const size_t n1 = (size_t)(p.I + 4) * H, n2 = (size_t)H * H3, n3 = (size_t)A * H;
@@ -134,6 +159,11 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       wsm[n1 + 2 * n2 + i] = a < A ? p.W2[(size_t)a * H + k] : 0.f;
     }
     (void)n3;
+    float* bs = wsm + n1 + 2 * n2 + (size_t)AQ * H;
+    for (int i = tid; i < H; i += FF_THREADS) bs[i] = p.b1[i];
+    for (int i = tid; i < H3; i += FF_THREADS) { bs[H + i] = p.bih[i]; bs[H + H3 + i] = p.bhh[i]; }
+    for (int i = tid; i < AQ; i += FF_THREADS) bs[H + 2 * H3 + i] = i < A ? p.b2[i] : 0.f;
+    B1 = bs; BIH = bs + H; BHH = bs + H + H3; B2 = bs + H + 2 * H3;
     W1T = wsm; WihT = wsm + n1; WhhT = wsm + n1 + n2; W2 = wsm + n1 + 2 * n2;
   }
   __syncthreads();
@@ -293,11 +323,11 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       // ---- phase B: fc1 ----
       for (int jb = 0; jb < H; jb += 64) {
         const int j0 = jb + tx * 4;
-        float acc[4][4];
+        f32x2 acc2[4][2];  // columns (0, 1) and (2, 3) of each row
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(p.b1 + rt[m] * tstride + j0));
-          acc[m][0] = b.x; acc[m][1] = b.y; acc[m][2] = b.z; acc[m][3] = b.w;
+          const ulonglong2 b = wload22<WS>(B1 + rt[m] * tstride + j0);
+          acc2[m][0] = b.x; acc2[m][1] = b.y;
         }
         const int K4 = (D + 3) & ~3;
         for (int typ = 0; typ < ntypes; ++typ)
@@ -310,16 +340,21 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           }
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            const float4 w = wload4<WS>(W1T + typ * tstride + (size_t)(k + kk) * H + j0);
+            const ulonglong2 w = wload22<WS>(W1T + typ * tstride + (size_t)(k + kk) * H + j0);
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
               const float xk = kk == 0 ? xv[m].x : kk == 1 ? xv[m].y : kk == 2 ? xv[m].z : xv[m].w;
-              acc[m][0] = fmaf(xk, w.x, acc[m][0]);
-              acc[m][1] = fmaf(xk, w.y, acc[m][1]);
-              acc[m][2] = fmaf(xk, w.z, acc[m][2]);
-              acc[m][3] = fmaf(xk, w.w, acc[m][3]);
+              const f32x2 xx = pack2(xk, xk);
+              acc2[m][0] = fma2(xx, w.x, acc2[m][0]);
+              acc2[m][1] = fma2(xx, w.y, acc2[m][1]);
             }
           }
+        }
+        float acc[4][4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          unpack2(acc2[m][0], acc[m][0], acc[m][1]);
+          unpack2(acc2[m][1], acc[m][2], acc[m][3]);
         }
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
@@ -342,72 +377,88 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       // ---- phase C: GRU cell ----
       for (int jb = 0; jb < H; jb += 64) {
         const int j0 = jb + tx * 4;
-        float ar[4][4], az[4][4], ai_[4][4], ah[4][4];
+        f32x2 ar2[4][2], az2[4][2], ai2[4][2], ah2[4][2];  // columns (0, 1) and (2, 3) of each row
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
-          const float* bih = p.bih + rt[m] * tstride;
-          const float* bhh = p.bhh + rt[m] * tstride;
-          const float4 bir = __ldg(reinterpret_cast<const float4*>(bih + j0));
-          const float4 biz = __ldg(reinterpret_cast<const float4*>(bih + H + j0));
-          const float4 bin = __ldg(reinterpret_cast<const float4*>(bih + 2 * H + j0));
-          const float4 bhr = __ldg(reinterpret_cast<const float4*>(bhh + j0));
-          const float4 bhz = __ldg(reinterpret_cast<const float4*>(bhh + H + j0));
-          const float4 bhn = __ldg(reinterpret_cast<const float4*>(bhh + 2 * H + j0));
-          {
-            ar[m][0] = bir.x + bhr.x; ar[m][1] = bir.y + bhr.y; ar[m][2] = bir.z + bhr.z; ar[m][3] = bir.w + bhr.w;
-            az[m][0] = biz.x + bhz.x; az[m][1] = biz.y + bhz.y; az[m][2] = biz.z + bhz.z; az[m][3] = biz.w + bhz.w;
-            ai_[m][0] = bin.x; ai_[m][1] = bin.y; ai_[m][2] = bin.z; ai_[m][3] = bin.w;
-            ah[m][0] = bhn.x; ah[m][1] = bhn.y; ah[m][2] = bhn.z; ah[m][3] = bhn.w;
-          }
+          const float* bih = BIH + rt[m] * tstride;
+          const float* bhh = BHH + rt[m] * tstride;
+          const float4 bir = wload4<WS>(bih + j0);
+          const float4 biz = wload4<WS>(bih + H + j0);
+          const float4 bin = wload4<WS>(bih + 2 * H + j0);
+          const float4 bhr = wload4<WS>(bhh + j0);
+          const float4 bhz = wload4<WS>(bhh + H + j0);
+          const float4 bhn = wload4<WS>(bhh + 2 * H + j0);
+          ar2[m][0] = pack2(bir.x + bhr.x, bir.y + bhr.y); ar2[m][1] = pack2(bir.z + bhr.z, bir.w + bhr.w);
+          az2[m][0] = pack2(biz.x + bhz.x, biz.y + bhz.y); az2[m][1] = pack2(biz.z + bhz.z, biz.w + bhz.w);
+          ai2[m][0] = pack2(bin.x, bin.y); ai2[m][1] = pack2(bin.z, bin.w);
+          ah2[m][0] = pack2(bhn.x, bhn.y); ah2[m][1] = pack2(bhn.z, bhn.w);
         }
-#pragma unroll 1
-        for (int tp = 0; tp < 2 * ntypes; ++tp) {
-          const int pass = tp & 1, typ = tp >> 1;
+        // (the pass is a compile-time constant of the loop body: chosen at run time, the products of the other pass'
+        // candidate accumulators would be issued and predicated off)
+        auto gemm_pass = [&](auto pass_c, int typ) {
+          constexpr int pass = decltype(pass_c)::value;
           const float* act = pass == 0 ? ys : (hs + cur * hbuf);
           const float* WT = (pass == 0 ? WihT : WhhT) + typ * tstride;
           const bool rnd = lowp && pass == 1;  // the hidden state is stored in fp32; its operand copy is rounded here
-          for (int k = 0; k < H; k += 4) {
-            float4 v[4];
+          // Software pipeline: the weights of k + 1 and the activations of the next four k are requested before the
+          // products of k are issued (indices past the end are clamped: loaded, never used), so that with two warps
+          // per scheduler a shared-memory latency is not waited for at every k.
+          auto load_act = [&](int k, float4 (&v)[4]) {
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
               v[m] = round4(*reinterpret_cast<const float4*>(act + (ty + 16 * m) * Hp + k), rnd);
               if (TYPED && rt[m] != typ) v[m] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
+          };
+          float4 v[4], vn[4];
+          load_act(0, v);
+          const float* wbase = WT + j0;
+          ulonglong2 wr = wload22<WS>(wbase), wz = wload22<WS>(wbase + H), wn = wload22<WS>(wbase + 2 * H);
+          for (int k = 0; k < H; k += 4) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-              const float* wrow = WT + (size_t)(k + kk) * H3 + j0;
-              const float4 wr = wload4<WS>(wrow);
-              const float4 wz = wload4<WS>(wrow + H);
-              const float4 wn = wload4<WS>(wrow + 2 * H);
+              const float* wrow = wbase + (size_t)min(k + kk + 1, H - 1) * H3;
+              const ulonglong2 wr_n = wload22<WS>(wrow), wz_n = wload22<WS>(wrow + H), wn_n = wload22<WS>(wrow + 2 * H);
+              if (kk == 1) load_act(min(k + 4, H - 4), vn);
 #pragma unroll
               for (int m = 0; m < 4; ++m) {
                 const float a = kk == 0 ? v[m].x : kk == 1 ? v[m].y : kk == 2 ? v[m].z : v[m].w;
-                ar[m][0] = fmaf(a, wr.x, ar[m][0]); ar[m][1] = fmaf(a, wr.y, ar[m][1]);
-                ar[m][2] = fmaf(a, wr.z, ar[m][2]); ar[m][3] = fmaf(a, wr.w, ar[m][3]);
-                az[m][0] = fmaf(a, wz.x, az[m][0]); az[m][1] = fmaf(a, wz.y, az[m][1]);
-                az[m][2] = fmaf(a, wz.z, az[m][2]); az[m][3] = fmaf(a, wz.w, az[m][3]);
+                const f32x2 aa = pack2(a, a);
+                ar2[m][0] = fma2(aa, wr.x, ar2[m][0]); ar2[m][1] = fma2(aa, wr.y, ar2[m][1]);
+                az2[m][0] = fma2(aa, wz.x, az2[m][0]); az2[m][1] = fma2(aa, wz.y, az2[m][1]);
                 if (pass == 0) {
-                  ai_[m][0] = fmaf(a, wn.x, ai_[m][0]); ai_[m][1] = fmaf(a, wn.y, ai_[m][1]);
-                  ai_[m][2] = fmaf(a, wn.z, ai_[m][2]); ai_[m][3] = fmaf(a, wn.w, ai_[m][3]);
+                  ai2[m][0] = fma2(aa, wn.x, ai2[m][0]); ai2[m][1] = fma2(aa, wn.y, ai2[m][1]);
                 } else {
-                  ah[m][0] = fmaf(a, wn.x, ah[m][0]); ah[m][1] = fmaf(a, wn.y, ah[m][1]);
-                  ah[m][2] = fmaf(a, wn.z, ah[m][2]); ah[m][3] = fmaf(a, wn.w, ah[m][3]);
+                  ah2[m][0] = fma2(aa, wn.x, ah2[m][0]); ah2[m][1] = fma2(aa, wn.y, ah2[m][1]);
                 }
               }
+              wr = wr_n; wz = wz_n; wn = wn_n;
             }
+#pragma unroll
+            for (int m = 0; m < 4; ++m) v[m] = vn[m];
           }
+        };
+#pragma unroll 1
+        for (int typ = 0; typ < ntypes; ++typ) {
+          gemm_pass(std::integral_constant<int, 0>(), typ);
+          gemm_pass(std::integral_constant<int, 1>(), typ);
         }
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
           const int r = ty + 16 * m;
           const float4 hp = *reinterpret_cast<const float4*>(hs + cur * hbuf + r * Hp + j0);
           const float hpv[4] = {hp.x, hp.y, hp.z, hp.w};
+          float ar[4], az[4], ai_[4], ah[4];
+          unpack2(ar2[m][0], ar[0], ar[1]); unpack2(ar2[m][1], ar[2], ar[3]);
+          unpack2(az2[m][0], az[0], az[1]); unpack2(az2[m][1], az[2], az[3]);
+          unpack2(ai2[m][0], ai_[0], ai_[1]); unpack2(ai2[m][1], ai_[2], ai_[3]);
+          unpack2(ah2[m][0], ah[0], ah[1]); unpack2(ah2[m][1], ah[2], ah[3]);
           float o[4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            const float rg = sigmoid_accurate(ar[m][c]);
-            const float zg = sigmoid_accurate(az[m][c]);
-            const float cand = tanhf(fmaf(rg, ah[m][c], ai_[m][c]));
+            const float rg = sigmoid_accurate(ar[c]);
+            const float zg = sigmoid_accurate(az[c]);
+            const float cand = tanhf(fmaf(rg, ah[c], ai_[c]));
             o[c] = fmaf(zg, hpv[c] - cand, cand);  // (1 - z) * cand + z * h
           }
           *reinterpret_cast<float4*>(hs + nxt * hbuf + r * Hp + j0) = make_float4(o[0], o[1], o[2], o[3]);
@@ -428,12 +479,13 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const int a = 16 * g + 4 * part + c;
-            q[g][c] = a < A ? __ldg(p.b2 + toff + a) : 0.f;
+            q[g][c] = a < A ? (WS ? B2[a] : __ldg(B2 + toff + a)) : 0.f;
           }
         const float* hv = hs + nxt * hbuf + r * Hp;
         if (WS) {
           const int AQ = (A + 3) & ~3;
           const float* wcol = W2 + 4 * part;  // W2T [k][AQ]
+#pragma unroll 4
           for (int k = 0; k < H; k += 4) {
             const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
 #pragma unroll
@@ -550,9 +602,16 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       }
       __syncthreads();
       // ---- phase F (second half): a closed episode starts from a zero hidden state and no last action ----
-      for (int r = tid >> 5; r < R; r += FF_THREADS / 32)  // a warp per row: the flag is read once, rows rarely reset
-        if (envs[r / n].reset)
+      {
+        // each warp looks after eight rows: one lane per row reads the flag, the vote says whether anything is to do
+        const int r8 = (tid >> 5) * 8 + (tid & 7);
+        uint32_t todo = __ballot_sync(0xFFFFFFFFu, (tid & 31) < 8 && r8 < R && envs[r8 / n].reset) & 0xFFu;
+        while (todo) {
+          const int r = (tid >> 5) * 8 + __ffs(todo) - 1;
+          todo &= todo - 1;
           for (int j = tid & 31; j < H; j += 32) hs[nxt * hbuf + r * Hp + j] = 0.f;
+        }
+      }
       if (tid < R && envs[tid / n].reset) la[tid] = -1;
       cur = nxt;
       __syncthreads();
