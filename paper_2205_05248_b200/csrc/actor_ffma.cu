@@ -251,6 +251,27 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       {
         const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
         const int nD = n * D;
+        const uint32_t inv_D = 0xFFFFFFFFu / (uint32_t)D + 1u, inv_nD = 0xFFFFFFFFu / (uint32_t)nD + 1u;
+        // A row's availability bytes as aligned words (up to three bytes on either side are read and dropped), all
+        // requested before the first is looked at: byte by byte, every load would wait for the one before it.
+        auto load_avail_row = [&](const uint8_t* av, uint32_t (&w)[10]) -> uint32_t {
+          const uintptr_t a0 = reinterpret_cast<uintptr_t>(av);
+          const uint32_t* wp = reinterpret_cast<const uint32_t*>(a0 & ~(uintptr_t)3);
+          const uint32_t sh = (uint32_t)(a0 & 3u), nw = (sh + (uint32_t)A + 3u) / 4u;
+#pragma unroll
+          for (int k = 0; k < 10; ++k) w[k] = (uint32_t)k < nw ? __ldg(wp + k) : 0u;
+          return sh;
+        };
+        auto mask_of = [&](const uint32_t (&w)[10], uint32_t sh) -> uint32_t {
+          unsigned long long bits = 0;
+#pragma unroll
+          for (int k = 0; k < 9; ++k) {
+            const uint32_t v = w[k];
+            const uint32_t nz = ((v | ((v & 0x7F7F7F7Fu) + 0x7F7F7F7Fu)) & 0x80808080u) >> 7;  // 0x01 per non-zero byte
+            bits |= (unsigned long long)((nz * 0x01020408u) >> 24 & 0xFu) << (4 * k);
+          }
+          return (uint32_t)(bits >> sh) & (A >= 32 ? 0xFFFFFFFFu : ((1u << A) - 1u));
+        };
         if (vec) {
           const int nv = R * D / 4;
 #pragma unroll
@@ -258,8 +279,8 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             const int idx = (tid + u * FF_THREADS) * 4;
             if (idx < nv * 4) {
               asm volatile("" : "+f"(pre[u].x), "+f"(pre[u].y), "+f"(pre[u].z), "+f"(pre[u].w));  // first use is here
-              const int r = idx / D, d = idx - r * D;
-              const int el = idx / nD;
+              const int r = (int)__umulhi((uint32_t)idx, inv_D), d = idx - r * D;  // (exact: idx < 2^16)
+              const int el = (int)__umulhi((uint32_t)idx, inv_nD);
               const float4 v = pre[u];
               *reinterpret_cast<float4*>(xs + r * Dp + d) = round4(v, lowp);
               const EnvSlot& es = envs[el];
@@ -282,28 +303,42 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             dst[idx - el * nD] = v;
           }
         }
+        if (s + 1 < p.T) {
+          // the next step's availability rows, rewards and end flags are first touches of their lines: ask for them
+          // now, so that the next phase A finds them in L2 instead of waiting for DRAM
+          if (tid < R) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.avail + (size_t)(s + 1) * p.avail_step_stride + ((size_t)e0 * n + tid) * A));
+          if (tid == FF_RMAX && !p.lagged) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.reward + (size_t)(s + 1) * p.env_step_stride + e0));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.done + (size_t)(s + 1) * p.env_step_stride + e0));
+          }
+        }
         if (tid < R) {
           const int el = tid / n, ai = tid - el * n;
           const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + ((size_t)e0 * n + tid) * A;
           const EnvSlot& es = envs[el];
           uint8_t* dst = p.ring + (size_t)es.slot * p.slot_stride + (size_t)es.pos * p.rl.rec_bytes +
                          p.rl.off_avail + ai * A;
-          uint32_t m = 0;
-          for (int a = 0; a < A; ++a) {
-            const uint8_t b = av[a];
-            if (b) m |= 1u << a;
-            if (es.ok) dst[a] = b;
+          uint32_t w[10];
+          const uint32_t sh = load_avail_row(av, w);
+          masks[tid] = mask_of(w, sh);
+          if (es.ok) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t v = __funnelshift_r(w[j], w[j + 1], 8u * sh);  // bytes 4 j .. 4 j + 3 of the row
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                if (4 * j + c < A) dst[4 * j + c] = (uint8_t)(v >> (8 * c));
+            }
           }
-          masks[tid] = m;
         }
         if (tid >= FF_RMAX && tid < FF_RMAX + R) {
           // The epsilon draw needs only the availability bytes (Algorithm 2 draws before it looks at Q): a second
           // set of threads reads them again and draws while the first set records them.
           const int r = tid - FF_RMAX, el = r / n, ai = r - el * n;
           const uint8_t* av = p.avail + (size_t)s * p.avail_step_stride + ((size_t)e0 * n + r) * A;
-          uint32_t m = 0;
-          for (int a = 0; a < A; ++a)
-            if (av[a]) m |= 1u << a;
+          uint32_t w[10];
+          const uint32_t sh = load_avail_row(av, w);
+          const uint32_t m = mask_of(w, sh);
           picks[r] = m ? draw_explore(m, eps, p.seed, t, (uint32_t)envs[el].eid, (uint32_t)ai) : -1;
         }
         if (tid < ne) {
