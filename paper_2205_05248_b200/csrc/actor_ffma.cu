@@ -27,15 +27,17 @@ constexpr int FF_PRE = 8;        // float4 registers per thread that hold the ne
 
 struct FfmaSmem {
   int Dp, Hp, wsmem;
-  size_t off_xs, off_ys, off_hs, off_pick, off_mask, off_la, off_env, off_w, w_floats, total;
+  size_t off_xs, off_ys, off_hs, off_pick, off_mask, off_la, off_env, off_small, off_w, w_floats, total;
 };
 
 // Floats of the weight image kept in shared memory when it fits (hidden size 64): the k-major matrices
-// W1T [I+4][H], WihT [H][3H], WhhT [H][3H] and W2T [H][A rounded up to 4], then the biases b1 [H], b_ih [3H],
-// b_hh [3H] and b2 [A rounded up to 4], in this order.
+// W1T [I+4][H], WihT [H][3H] and WhhT [H][3H], in this order.
 __host__ __device__ inline size_t ffma_weight_floats(int n, int D, int A, int H) {
-  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H + (size_t)((A + 3) & ~3) * (H + 1) + 7 * (size_t)H;
+  return (size_t)(D + n + A + 4) * H + 2 * (size_t)H * 3 * H;
 }
+// Floats of the small image that a shared network always keeps in shared memory: W2T [H][A rounded up to 4], then the
+// biases b1 [H], b_ih [3H], b_hh [3H] and b2 [A rounded up to 4].
+__host__ __device__ inline size_t ffma_small_floats(int A, int H) { return (size_t)((A + 3) & ~3) * (H + 1) + 7 * (size_t)H; }
 
 __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H) {
   FfmaSmem s;
@@ -51,6 +53,7 @@ __host__ __device__ inline FfmaSmem ffma_smem_layout(int n, int D, int A, int H)
   s.off_mask = o; o += sizeof(uint32_t) * FF_RMAX;
   s.off_la = o; o += sizeof(int32_t) * FF_RMAX;
   s.off_env = o; o += 40 * FF_RMAX;  // per-environment scratch: see EnvSlot
+  s.off_small = o; o += sizeof(float) * ffma_small_floats(A, H);
   s.off_w = o;
   s.w_floats = ffma_weight_floats(n, D, A, H);
   s.wsmem = (o + sizeof(float) * s.w_floats <= 227 * 1024) ? 1 : 0;  // resident weights if they fit
@@ -146,27 +149,31 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
   unsigned long long c_steps = 0, c_explore = 0, c_noavail = 0, c_episodes = 0, c_trunc = 0;
   uint32_t st_bits = 0;
 
-  for (int i = tid; i < (int)(sl.off_w / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;
+  for (int i = tid; i < (int)(sl.off_small / 4); i += FF_THREADS) reinterpret_cast<uint32_t*>(smem)[i] = 0;  // (the images follow)
   // weight pointers: the resident copy, or the k-major global arrays
   const float *W1T = p.W1T, *WihT = p.WihT, *WhhT = p.WhhT, *W2 = p.W2;
   const float *B1 = p.b1, *BIH = p.bih, *BHH = p.bhh, *B2 = p.b2;  // (a phase that starts with a load from global memory waits for it every step)
-  if (WS) {
-    float* wsm = reinterpret_cast<float*>(smem + sl.off_w);
-    const size_t n1 = (size_t)(p.I + 4) * H, n2 = (size_t)H * H3, n3 = (size_t)A * H;
-    for (size_t i = tid; i < n1; i += FF_THREADS) wsm[i] = p.W1T[i];
-    for (size_t i = tid; i < n2; i += FF_THREADS) { wsm[n1 + i] = p.WihT[i]; wsm[n1 + n2 + i] = p.WhhT[i]; }
+  constexpr bool SS = !TYPED;  // a shared network: W2 (transposed) and the biases are resident whatever the hidden size
+  if (SS) {
+    float* ssm = reinterpret_cast<float*>(smem + sl.off_small);
     const int AQ = (A + 3) & ~3;  // W2 transposed: the actions of one k side by side, padded with zeros
     for (size_t i = tid; i < (size_t)AQ * H; i += FF_THREADS) {
       const int k = (int)(i / AQ), a = (int)(i - (size_t)k * AQ);
-      wsm[n1 + 2 * n2 + i] = a < A ? p.W2[(size_t)a * H + k] : 0.f;
+      ssm[i] = a < A ? p.W2[(size_t)a * H + k] : 0.f;
     }
-    (void)n3;
-    float* bs = wsm + n1 + 2 * n2 + (size_t)AQ * H;
+    float* bs = ssm + (size_t)AQ * H;
     for (int i = tid; i < H; i += FF_THREADS) bs[i] = p.b1[i];
     for (int i = tid; i < H3; i += FF_THREADS) { bs[H + i] = p.bih[i]; bs[H + H3 + i] = p.bhh[i]; }
     for (int i = tid; i < AQ; i += FF_THREADS) bs[H + 2 * H3 + i] = i < A ? p.b2[i] : 0.f;
     B1 = bs; BIH = bs + H; BHH = bs + H + H3; B2 = bs + H + 2 * H3;
-    W1T = wsm; WihT = wsm + n1; WhhT = wsm + n1 + n2; W2 = wsm + n1 + 2 * n2;
+    W2 = ssm;
+  }
+  if (WS) {
+    float* wsm = reinterpret_cast<float*>(smem + sl.off_w);
+    const size_t n1 = (size_t)(p.I + 4) * H, n2 = (size_t)H * H3;
+    for (size_t i = tid; i < n1; i += FF_THREADS) wsm[i] = p.W1T[i];
+    for (size_t i = tid; i < n2; i += FF_THREADS) { wsm[n1 + i] = p.WihT[i]; wsm[n1 + n2 + i] = p.WhhT[i]; }
+    W1T = wsm; WihT = wsm + n1; WhhT = wsm + n1 + n2;
   }
   __syncthreads();
 
@@ -363,7 +370,7 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         f32x2 acc2[4][2];  // columns (0, 1) and (2, 3) of each row
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
-          const ulonglong2 b = wload22<WS>(B1 + rt[m] * tstride + j0);
+          const ulonglong2 b = wload22<SS>(B1 + rt[m] * tstride + j0);
           acc2[m][0] = b.x; acc2[m][1] = b.y;
         }
         const int K4 = (D + 3) & ~3;
@@ -401,9 +408,9 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           const float4 wid = wload4<WS>(W1T + rt[m] * tstride + (size_t)(D + ai) * H + j0);
           float4 o = make_float4(acc[m][0] + wid.x, acc[m][1] + wid.y, acc[m][2] + wid.z, acc[m][3] + wid.w);
           const int last = la[r];
-          if (last >= 0) {
-            const float4 wl = wload4<WS>(W1T + rt[m] * tstride + (size_t)(D + n + last) * H + j0);
-            o.x += wl.x; o.y += wl.y; o.z += wl.z; o.w += wl.w;
+          {  // (loaded whether or not there is a last action - row 0 then, dropped: a load under a condition is waited for)
+            const float4 wl = wload4<WS>(W1T + rt[m] * tstride + (size_t)(D + n + max(last, 0)) * H + j0);
+            if (last >= 0) { o.x += wl.x; o.y += wl.y; o.z += wl.z; o.w += wl.w; }
           }
           o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
           if (lowp) { o.x = bf16_round(o.x); o.y = bf16_round(o.y); o.z = bf16_round(o.z); o.w = bf16_round(o.w); }
@@ -420,12 +427,12 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
         for (int m = 0; m < 4; ++m) {
           const float* bih = BIH + rt[m] * tstride;
           const float* bhh = BHH + rt[m] * tstride;
-          const float4 bir = wload4<WS>(bih + j0);
-          const float4 biz = wload4<WS>(bih + H + j0);
-          const float4 bin = wload4<WS>(bih + 2 * H + j0);
-          const float4 bhr = wload4<WS>(bhh + j0);
-          const float4 bhz = wload4<WS>(bhh + H + j0);
-          const float4 bhn = wload4<WS>(bhh + 2 * H + j0);
+          const float4 bir = wload4<SS>(bih + j0);
+          const float4 biz = wload4<SS>(bih + H + j0);
+          const float4 bin = wload4<SS>(bih + 2 * H + j0);
+          const float4 bhr = wload4<SS>(bhh + j0);
+          const float4 bhz = wload4<SS>(bhh + H + j0);
+          const float4 bhn = wload4<SS>(bhh + 2 * H + j0);
           ar2[m][0] = pack2(bir.x + bhr.x, bir.y + bhr.y); ar2[m][1] = pack2(bir.z + bhr.z, bir.w + bhr.w);
           az2[m][0] = pack2(biz.x + bhz.x, biz.y + bhz.y); az2[m][1] = pack2(biz.z + bhz.z, biz.w + bhz.w);
           ai2[m][0] = pack2(bin.x, bin.y); ai2[m][1] = pack2(bin.z, bin.w);
@@ -518,10 +525,10 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const int a = 16 * g + 4 * part + c;
-            q[g][c] = a < A ? (WS ? B2[a] : __ldg(B2 + toff + a)) : 0.f;
+            q[g][c] = a < A ? (SS ? B2[a] : __ldg(B2 + toff + a)) : 0.f;
           }
         const float* hv = hs + nxt * hbuf + r * Hp;
-        if (WS) {
+        if (SS) {
           const int AQ = (A + 3) & ~3;
           const float* wcol = W2 + 4 * part;  // W2T [k][AQ]
           // Unconditional loads, so that the four k of a pass are requested together (a load under a per-thread
@@ -563,21 +570,27 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             }
           }
         } else {
+          // weights from global memory, W2 [A][H]: the loads are unconditional (the action index clamped to A - 1; the
+          // sums of actions beyond A are never used), so that those of one k-group are requested together
+          const bool two = A > 16;
           for (int k = 0; k < H; k += 4) {
             const float4 v = round4(*reinterpret_cast<const float4*>(hv + k), lowp);
+            float4 w[2][4];
 #pragma unroll
             for (int g = 0; g < 2; ++g)
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const int a = 16 * g + 4 * part + c;
-                if (a < A) {
-                  const float4 w = wload4<WS>(W2 + toff + (size_t)a * H + k);
-                  q[g][c] = fmaf(v.x, w.x, q[g][c]);
-                  q[g][c] = fmaf(v.y, w.y, q[g][c]);
-                  q[g][c] = fmaf(v.z, w.z, q[g][c]);
-                  q[g][c] = fmaf(v.w, w.w, q[g][c]);
+              for (int c = 0; c < 4; ++c)
+                if (g == 0 || two) w[g][c] = wload4<false>(W2 + toff + (size_t)min(16 * g + 4 * part + c, A - 1) * H + k);
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                if (g == 0 || two) {
+                  q[g][c] = fmaf(v.x, w[g][c].x, q[g][c]);
+                  q[g][c] = fmaf(v.y, w[g][c].y, q[g][c]);
+                  q[g][c] = fmaf(v.z, w[g][c].z, q[g][c]);
+                  q[g][c] = fmaf(v.w, w[g][c].w, q[g][c]);
                 }
-              }
           }
         }
         // greedy rule: m = max over available, thr = m - 1e-4f, lowest available a with Q >= thr (a NaN never
