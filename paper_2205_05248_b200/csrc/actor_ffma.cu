@@ -11,7 +11,8 @@
 //   B  fc1 + one-hot column gathers + ReLU                       (register-tiled 4 rows x 4 columns)
 //   C  GRU cell: both gate GEMMs, gate math, new hidden state    (same tiling, 64 accumulators)
 //   D  fc2, masked greedy choice, ring/trace writes              (four threads per row, Q in registers)
-//   F  reward/done, episode bookkeeping, hidden-state reset      (one thread per environment, then a warp per row)
+//   F  reward/done, episode bookkeeping                          (one thread per environment); the hidden-state reset
+//      of closed episodes shares the next step's phase A (a warp per eight rows)
 // Weights are read through the read-only path from k-major copies, so a warp's load of four output
 // columns for one k is one contiguous 256-byte segment.
 #include <type_traits>
@@ -251,12 +252,27 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
       __syncthreads();
     }
 
+    // A closed episode starts from a zero hidden state and no last action.  Needs the flags of the bookkeeping phase
+    // and touches neither what staging reads nor what it writes, so it shares a phase with the next step's staging.
+    auto reset_closed = [&](int buf) {
+      // each warp looks after eight rows: one lane per row reads the flag, the vote says whether anything is to do
+      const int r8 = (tid >> 5) * 8 + (tid & 7);
+      uint32_t todo = __ballot_sync(0xFFFFFFFFu, (tid & 31) < 8 && r8 < R && envs[r8 / n].reset) & 0xFFu;
+      while (todo) {
+        const int r = (tid >> 5) * 8 + __ffs(todo) - 1;
+        todo &= todo - 1;
+        for (int j = tid & 31; j < H; j += 32) hs[buf * hbuf + r * Hp + j] = 0.f;
+      }
+      if (tid < R && envs[tid / n].reset) la[tid] = -1;
+    };
+
     for (int s = 0; s < p.T; ++s) {
       const uint32_t t = p.t0 + (uint32_t)s;
       const float eps = eps_at(p, t);
       const int nxt = cur ^ 1;
 
       // ---- phase A ----
+      if (s > 0) reset_closed(cur);  // (the previous step's)
       {
         const float* src = p.obs + (size_t)s * p.obs_step_stride + (size_t)e0 * n * D;
         const int nD = n * D;
@@ -354,7 +370,6 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
           EnvSlot& es = envs[tid];
           es.reward = p.lagged ? 0.f : p.reward[(size_t)s * p.env_step_stride + e0 + tid];
           es.done = (!p.lagged && p.done[(size_t)s * p.env_step_stride + e0 + tid]) ? 1 : 0;
-          es.reset = 0;
           if (es.ok && es.pos == 0) {  // an episode opens in this slot
             p.slot_epid[es.slot] = es.epc * (long long)p.E + es.eid;
             p.slot_len[es.slot] = 0;
@@ -671,25 +686,15 @@ __global__ void __launch_bounds__(FF_THREADS, 1) actor_ffma_kernel(const __grid_
             es.reset = 1;
           } else {
             es.pos += 1;
+            es.reset = 0;
           }
         }
       }
-      __syncthreads();
-      // ---- phase F (second half): a closed episode starts from a zero hidden state and no last action ----
-      {
-        // each warp looks after eight rows: one lane per row reads the flag, the vote says whether anything is to do
-        const int r8 = (tid >> 5) * 8 + (tid & 7);
-        uint32_t todo = __ballot_sync(0xFFFFFFFFu, (tid & 31) < 8 && r8 < R && envs[r8 / n].reset) & 0xFFu;
-        while (todo) {
-          const int r = (tid >> 5) * 8 + __ffs(todo) - 1;
-          todo &= todo - 1;
-          for (int j = tid & 31; j < H; j += 32) hs[nxt * hbuf + r * Hp + j] = 0.f;
-        }
-      }
-      if (tid < R && envs[tid / n].reset) la[tid] = -1;
       cur = nxt;
       __syncthreads();
     }
+    reset_closed(cur);  // (the last step's)
+    __syncthreads();
 
     // ---- tile store ----
     for (int idx = tid; idx < R * H; idx += FF_THREADS) {
