@@ -316,8 +316,8 @@ int marl_actor_create(const marl_actor_config_t* cfg, marl_actor_t** out) {
   }
   // Kernel choice.  fp32 precision: the CUDA-core kernel (tensor cores cannot meet its 1e-5 tolerance).  bf16: a
   // tensor-core kernel wherever the shape is supported, at every batch size - timed on the same rollouts from 24
-  // rows to 16384 (`bench.py --crossover`), one 128-row tcgen05 tile takes 3.4-4.6 us per
-  // environment step against 25-29 us for the CUDA-core kernel's 64-row tiles, so there is no batch size at which
+  // rows to 16384 (`bench.py --crossover`), one 128-row tcgen05 tile takes 3.3-5.2 us per
+  // environment step against 18-21 us for the CUDA-core kernel's 64-row tiles, so there is no batch size at which
   // the CUDA cores win.
   // (the two-tile kernel is never the automatic choice: measured at workload 5 it is slower than the pipelined kernel -
   // 8.4 ms against 6.15 ms per 64-step rollout - because with the epilogue threads busy all the time the converter
