@@ -118,7 +118,7 @@ __device__ __forceinline__ float4 round4(float4 v, bool lowp) {
 // TYPED: one network per unit type (heterogeneous teams).  The tile's rows mix types, and a thread's register tile
 // shares each weight value among its four rows, so the three products run once per type on that type's image with
 // the operand of every row of another type replaced by zero: fma(0, w, acc) leaves acc as it is, so a row
-// accumulates exactly the products of its own network.  Biases, the one-hot columns and fc2 (one row per thread)
+// accumulates exactly the products of its own network.  Biases, the one-hot columns and fc2 (four threads per row)
 // read the row's own image directly.  The images are read through the read-only path (they do not fit shared memory
 // together).
 // LOWP: operands rounded to bf16 (a template parameter: as a run-time flag it put a branch behind every operand
